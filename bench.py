@@ -2,21 +2,30 @@
 """Benchmark of the Parallax decode forward on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C3] [--impl ours|reference]
+                    [--shard-keys]
 
 One step = one full decode call (one fused launch: split kernel whose last CTA per stream merges) over one batch of the
 named synthetic workload.  Prints ONE JSON line (rank 0).  The headline value is
 achieved KV-read bandwidth (algorithmic K+V bytes / device time, summed over
 GPUs); ms_per_step carries the latency (us/call = 1000 * ms_per_step).
 
-Under torchrun every rank runs the same per-GPU workload on its own seeded
-inputs (weak scaling: sequences are independent, there is no data-path
-collective); the time is the maximum over ranks.
+Several GPUs: `--gpus N` without a torchrun environment starts N ranks itself (one process per GPU,
+NCCL); under torchrun (WORLD_SIZE set) the process is one of the ranks.  Two partitions of the path:
+  default       every rank runs the same per-GPU workload on its own seeded sequences (weak scaling:
+                sequences are independent, there is no data-path collective);
+  --shard-keys  ONE batch whose keys are divided among the ranks (strong scaling): every rank turns
+                its slice of each context into partial states, the records are all-gathered, every
+                rank merges them.
+The time is the slowest rank's; a block of exactly K steps is timed between barriers and repeated
+until at least 200 ms of device time have been measured (median block reported, spread beside it).
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
+import subprocess
 import sys
 import threading
 import time
@@ -33,18 +42,30 @@ from paper_2605_29157_b200 import workloads as wl  # noqa: E402
 METRIC = "parallax_decode_kv_read_bandwidth"
 KV_LAYOUT = ["contiguous [B,Hkv,T,D]"]
 UNIT = "TB/s"
-NCU_TRAFFIC_FP8 = {"C3": 2 * 540_800_000}   # profiles/plx_decode_kernel_fp8_C3.md (B=32 capture x 2)
 L2_BYTES = 126 * 1024 * 1024
+MIN_TIMED_MS = 200.0     # device time every reported number rests on, whatever --steps is
+MAX_BLOCKS = 4000
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the main kernel, from the ncu
-# captures summarised under profiles/ (None = no capture for that workload).
-NCU_TRAFFIC_BYTES = {"C3": 2_155_300_000,   # profiles/plx_decode_kernel_C3.md (B=32 capture x 2)
-                     "C4": 1_077_300_000,   # profiles/plx_decode_kernel_C4.md (full size)
-                     "C6": 2 * 541_600_000,  # profiles/plx_decode_kernel_C6_d64.md (B=32 capture x 2)
-                     # tensor-bound kernels, captured on a reduced batch and scaled by the batch ratio
-                     # (sequences are independent, so DRAM traffic grows in proportion):
-                     "P1": 8 * 51_000_000,  # profiles/plx_prefill_kernel_P1.md (B=1 capture: 50.4 MB read + 0.6 MB written)
-                     "T1": 4 * 513_000_000}  # profiles/plx_bwd_kernels_T1.md (B=2 capture: row 175 + column 232 + prep 106 MB)
+# DRAM traffic of the dominant kernel per launch (dram__bytes_read.sum + dram__bytes_write.sum of one
+# ncu capture).  NOT measured in this run: each entry says which kernel instantiation and which capture
+# size it comes from and how it was scaled to a full launch (sequences are independent, so traffic grows
+# in proportion to the batch).  An entry goes stale when its kernel changes; the bench line carries the
+# provenance string beside the number.
+NCU_TRAFFIC = {
+    "C2": (134_600_000, "plx_decode_kernel<128,2,3,2>, full-size capture (cache sets rotated, so reads miss L2)"),
+    "C3": (2_155_300_000, "plx_decode_kernel<128,2,3,2>, capture at B=32 scaled x2"),
+    "C4": (1_077_300_000, "plx_decode_kernel<128,2,3,2>, full-size capture"),
+    "C6": (2 * 541_600_000, "plx_decode_kernel<64,2,2,4>, capture at B=32 scaled x2"),
+    "P1": (8 * 51_000_000, "plx_prefill_kernel<128>, capture at B=1 scaled x8"),
+    "T1": (4 * 513_000_000, "plx_bwd_prep/row/col kernels, capture at B=2 scaled x4"),
+}
+NCU_TRAFFIC_FP8 = {"C3": (2 * 540_800_000, "plx_decode_kernel<128,2,2,4,fp8>, capture at B=32 scaled x2")}
+
+
+def ncu_traffic(name, fp8=False):
+    """(bytes per launch or None, provenance or None) for a workload's dominant kernel."""
+    entry = (NCU_TRAFFIC_FP8 if fp8 else NCU_TRAFFIC).get(name)
+    return (entry[0], "ncu capture, not measured in this run: " + entry[1]) if entry else (None, None)
 
 
 def measured_peaks():
@@ -59,11 +80,13 @@ def measured_peaks():
 # clocks sampled during the timed regions (read-only NVML queries)
 # ----------------------------------------------------------------------------------------------
 class ClockSampler:
+    """SM clock and clock-event reasons polled every 5 ms through NVML (read-only queries) while `active`
+    is set.  `mark()` / `summary(since)` give the statistics of one timed region."""
     REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
                0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting"}
 
     def __init__(self, device_index: int):
-        self.samples, self.reason_bits = [], 0
+        self.samples, self.bits = [], []
         self.active = threading.Event()
         self.stop = threading.Event()
         self.handle, self.max_mhz = None, None
@@ -92,19 +115,85 @@ class ClockSampler:
                     except Exception:
                         bits = int(self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
                     self.samples.append(mhz)
-                    self.reason_bits |= bits
+                    self.bits.append(bits)
                 except Exception:
                     pass
-            time.sleep(0.01)
+            time.sleep(0.005)
 
-    def summary(self):
+    def mark(self) -> int:
+        return len(self.samples)
+
+    def summary(self, since: int = 0):
+        samples, bits = self.samples[since:], self.bits[since:]
+        if not samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        seen = 0
+        for x in bits:
+            seen |= x
+        reasons = [name for bit, name in self.REASONS.items() if seen & bit]
+        return {"sm_mhz": float(np.median(samples)), "sm_min_mhz": float(min(samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": reasons, "samples": len(samples)}
+
+    def close(self):
         self.stop.set()
         self.thread.join(timeout=1.0)
-        if not self.samples:
-            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
-        reasons = [name for bit, name in self.REASONS.items() if self.reason_bits & bit]
-        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz, "reasons": reasons,
-                "samples": len(self.samples)}
+
+
+# ----------------------------------------------------------------------------------------------
+# timed regions
+# ----------------------------------------------------------------------------------------------
+class BlockTimer:
+    """Times blocks of exactly `steps` calls with CUDA events on the launching stream, each block between a
+    barrier + device synchronisation on both sides, the slowest rank's time taken per block; blocks are
+    repeated until `min_ms` of device time have been measured (the same count on every rank: the
+    decision uses the reduced times).  Reports the median block."""
+
+    def __init__(self, stream, sampler, world=1, device="cuda"):
+        self.stream, self.sampler, self.world, self.device = stream, sampler, world, device
+
+    def barrier(self):
+        if self.world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    def block(self, fn, steps, offset=0):
+        self.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(self.stream)
+        for i in range(steps):
+            fn(offset + i)
+        e1.record(self.stream)
+        self.barrier()
+        return max_over_ranks(e0.elapsed_time(e1), self.world, self.device)
+
+    def run(self, fn, steps, min_ms=MIN_TIMED_MS):
+        """-> dict: ms_per_step (median block / steps), blocks, ms_total, spread (min, max of the blocks'
+        ms per step) and the clock summary of the region."""
+        since = self.sampler.mark() if self.sampler else 0
+        if self.sampler:
+            self.sampler.active.set()
+        times, total = [], 0.0
+        while (total < min_ms and len(times) < MAX_BLOCKS) or not times:
+            t = self.block(fn, steps, offset=len(times) * steps)
+            times.append(t)
+            total += t
+        if self.sampler:
+            self.sampler.active.clear()
+        per = np.array(times) / steps
+        return {"ms_per_step": float(np.median(per)), "blocks": len(times), "ms_total": float(total),
+                "ms_per_step_min": float(per.min()), "ms_per_step_max": float(per.max()),
+                "clocks": self.sampler.summary(since) if self.sampler else None}
+
+
+def timing_note(t):
+    return {"timed_blocks": t["blocks"], "device_ms_timed": round(t["ms_total"], 2),
+            "us_per_step_min": round(t["ms_per_step_min"] * 1e3, 2), "us_per_step_max": round(t["ms_per_step_max"] * 1e3, 2)}
+
+
+def free_port() -> int:
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
 
 
 # ----------------------------------------------------------------------------------------------
@@ -178,6 +267,37 @@ def max_over_ranks(ms: float, world: int, device="cpu") -> float:
 def whole_job_value(bytes_per_rank: int, world: int, ms_per_step: float) -> float:
     """TB/s over all ranks: every rank moved bytes_per_rank in the slowest rank's time."""
     return bytes_per_rank * world / (ms_per_step * 1e-3) / 1e12
+
+
+def read_probe(dev, stream, sampler):
+    """Read-only streaming bandwidth of this GPU, measured in this run with the library's own probe kernel:
+    2 GiB buffers, two of them read alternately (4 GiB between two reads of a byte vs 0.123 GiB of L2), each
+    variant timed for >= 100 ms.  Returns the per-variant GB/s and the best of them: the ceiling of a kernel
+    that only reads."""
+    from paper_2605_29157_b200 import binding as plx
+    nbytes = 2 << 30
+    bufs = [torch.empty(nbytes // 4, dtype=torch.int32, device=dev).random_() for _ in range(2)]
+    sink = torch.empty(plx.PLX_PROBE_SINK_BYTES, dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    timer = BlockTimer(stream, sampler)
+    variants = {
+        "vector_loads_8_ctas_per_sm": (plx.PLX_PROBE_VECTOR_LOADS, 0),
+        "vector_loads_64KiB_per_cta": (plx.PLX_PROBE_VECTOR_LOADS, nbytes // 65536),
+        "bulk_copies_2_ctas_per_sm": (plx.PLX_PROBE_BULK_COPIES, 0),
+        "bulk_copies_1MiB_per_cta": (plx.PLX_PROBE_BULK_COPIES, nbytes >> 20),
+    }
+    out = {}
+    for name, (mode, ctas) in variants.items():
+        def call(i, mode=mode, ctas=ctas):
+            plx.parallax_read_probe(bufs[i % 2], sink, mode, ctas, status, stream)
+        for i in range(3):
+            call(i)
+        t = timer.run(call, 10, min_ms=100.0)
+        out[name] = round(nbytes / (t["ms_per_step"] * 1e-3) / 1e9, 1)
+    assert int(status.item()) == 0, "read probe: a bounded wait ran out"
+    best = max(out, key=out.get)
+    return {"GBps": out, "best": best, "peak": out[best], "bytes_per_launch": nbytes,
+            "l2_policy": "two 2 GiB buffers read alternately"}
 
 
 def describe(cfg, seqlens_host, nsets, chunk, ns):
@@ -258,28 +378,12 @@ def run_ours(args, rank, world, local_rank):
         else:
             plx.parallax_decode_fwd_ex(x["q"], x["r"], x["k"], x["v"], x["seqlens"], out, cfg.scale, ws, args.splits, st)
 
-    def barrier():
-        if world > 1:
-            torch.distributed.barrier()
-        torch.cuda.synchronize()
-
-    def timed(fn, steps):
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        sampler.active.set()
-        e0.record(stream)
-        for i in range(steps):
-            fn(i)
-        e1.record(stream)
-        barrier()
-        sampler.active.clear()
-        return max_over_ranks(e0.elapsed_time(e1), world, dev)
-
     sampler = ClockSampler(local_rank)
+    timer = BlockTimer(stream, sampler, world, dev)
     for i in range(args.warmup):
         step(i)
-    ms_total = timed(step, args.steps)
-    ms_per_step = ms_total / args.steps
+    t_call = timer.run(step, args.steps)
+    ms_per_step = t_call["ms_per_step"]
     # one launch per call, except steps the library hands to the tensor-core kernel (more than eight rows per KV head)
     launches_per_step = tensor_core_launches(cfg, Lq, sms) if cfg.G * Lq > 8 and not (args.fp8_kv or args.page_size) else 1
     value = whole_job_value(kv_bytes, world, ms_per_step)
@@ -301,16 +405,23 @@ def run_ours(args, rank, world, local_rank):
                                                 chunk, ns, None, stream)
     for i in range(max(3, args.warmup)):
         main_only(i)
-    ms_kernel = timed(main_only, args.steps) / args.steps
+    t_kernel = timer.run(main_only, args.steps)
+    ms_kernel = t_kernel["ms_per_step"]
     peak, peak_src = measured_peaks()
     achieved = kv_bytes / (ms_kernel * 1e-3) / 1e9
+    traffic, traffic_src = ((None, None) if (args.page_size or Lq > 1 or args.batch or args.splits) else
+                            ncu_traffic(cfg.name, args.fp8_kv))
     roofline = {"bound": "hbm", "kernel": "plx_decode_kernel", "achieved": round(achieved, 1), "peak": peak,
-                "peak_source": f"{peak_src} copy bandwidth", "unit": "GB/s", "frac": round(achieved / peak, 4),
+                "peak_source": f"{peak_src} copy bandwidth (read + write)", "unit": "GB/s", "frac": round(achieved / peak, 4),
                 "frac_of_8TBps_nominal": round(achieved / 8000.0, 4),
                 "us_per_launch": round(ms_kernel * 1e3, 2),
                 "algorithmic_bytes_per_launch": kv_bytes,
-                "traffic": (NCU_TRAFFIC_FP8.get(cfg.name) if args.fp8_kv else
-                            None if (args.page_size or Lq > 1) else NCU_TRAFFIC_BYTES.get(cfg.name))}
+                "traffic": traffic, "traffic_source": traffic_src, **timing_note(t_kernel)}
+    if rank == 0 and not args.no_read_probe:
+        probe = read_probe(dev, stream, sampler)
+        roofline["peak_read_probe"] = probe["peak"]
+        roofline["frac_of_read_probe"] = round(achieved / probe["peak"], 4)
+        roofline["read_probe"] = probe
 
     # end to end through the host-buffer entry point: q, r from pinned host memory, out to host
     qh = [x["q"].cpu().pin_memory() for x in sets]
@@ -331,7 +442,8 @@ def run_ours(args, rank, world, local_rank):
     e2e_steps = max(10, args.steps // 4)
     for i in range(3):
         e2e_step(i)
-    ms_e2e = timed(e2e_step, e2e_steps) / e2e_steps
+    t_e2e = timer.run(e2e_step, e2e_steps)
+    ms_e2e = t_e2e["ms_per_step"]
     n_qr = cfg.B * cfg.Hq * Lq * cfg.D * 2
     e2e = {"value": round(whole_job_value(kv_bytes, world, ms_e2e), 4), "unit": UNIT,
            "us_per_call": round(ms_e2e * 1e3, 2), "h2d_bytes_per_step": 2 * n_qr, "d2h_bytes_per_step": n_qr,
@@ -340,8 +452,8 @@ def run_ours(args, rank, world, local_rank):
                     if (args.page_size or args.fp8_kv or Lq > 1) else
                     "q and r read from pinned host memory and the output written to pinned host memory every step "
                     "(by the library's staging kernel and by the attention kernel itself, over the host link); ") +
-                   "the KV cache is device-resident state of a decode step"}
-    clocks = sampler.summary()
+                   "the KV cache is device-resident state of a decode step", **timing_note(t_e2e)}
+    clocks = t_call["clocks"]
 
     result = {
         "metric": METRIC, "value": round(value, 4), "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -349,7 +461,10 @@ def run_ours(args, rank, world, local_rank):
         "us_per_call_graph_replay": round(us_graph, 2),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp16 products on an e4m3 cache" if args.fp8_kv else "bf16",
         "data": "synthetic", "config": describe(cfg, seqlens_host, nsets, chunk, ns),
-        "roofline": roofline, "e2e": e2e, "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+        "roofline": roofline, "e2e": e2e, "gpu_launches": launches_per_step * args.steps * t_call["blocks"],
+        "clocks": clocks, "timing": {"protocol": f"blocks of exactly {args.steps} steps between barriers, repeated until "
+                                                 f">= {MIN_TIMED_MS:.0f} ms of device time; median block reported",
+                                     **timing_note(t_call)},
     }
     if args.fp8_kv:   # the e4m3 variant plans its own splits inside the library
         result["config"]["chunk_len"] = result["config"]["num_splits"] = "planned inside the library for the e4m3 variant"
@@ -360,11 +475,15 @@ def run_ours(args, rank, world, local_rank):
     if rank == 0 and world == 1 and args.all_configs and not args.fp8_kv and Lq == 1:
         del sets
         torch.cuda.empty_cache()
-        result["other_configs"] = {n: quick_config(n) for n in sorted(wl.CONFIGS) if n != args.workload}
+        read_peak = roofline.get("peak_read_probe")
+        result["other_configs"] = {n: quick_config(n, sampler, read_peak) for n in sorted(wl.CONFIGS) if n != args.workload}
+        result["other_workloads"] = {n: quick_tensor_workload(n, local_rank) for n in ("P2", "T1")}
     if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.fp8_kv and Lq == 1:
         secs, nbytes, threads, desc = oracle_sample_time(cfg, x0, seqlens_host, args.cpu_seconds)
         result["cpu_baseline"] = {"value": round(nbytes / secs / 1e12, 8), "unit": UNIT, "cores": threads,
-                                  "kind": "oracle", "sample": desc, "seconds": round(secs, 2)}
+                                  "kind": "oracle", "sample": desc, "seconds": round(secs, 2),
+                                  "single_thread_C2": single_thread_oracle_c2()}
+    sampler.close()
     return result
 
 
@@ -398,9 +517,10 @@ def graph_replay_us(step, nsets, reps=5):
     return e0.elapsed_time(e1) / (reps * per_graph) * 1e3
 
 
-def quick_config(name, steps=60, warmup=5):
-    """Short device-timed run of one decode configuration (library plan, L2-cold by rotating cache sets):
-    us per call, KV-read TB/s, fraction of the measured copy bandwidth."""
+def quick_config(name, sampler, read_peak=None, steps=20, warmup=5):
+    """Device-timed run of one decode configuration (library plan, L2-cold by rotating cache sets, blocks of
+    `steps` calls repeated until >= 200 ms of device time): us per call, KV-read TB/s, its fractions of the
+    measured copy bandwidth, of this run's read-only probe and of 8 TB/s, and the clocks of its own region."""
     from paper_2605_29157_b200 import binding as plx
     cfg = wl.CONFIGS[name]
     kv_set_bytes = cfg.B * cfg.Hkv * cfg.T_max * cfg.D * 4
@@ -418,19 +538,45 @@ def quick_config(name, steps=60, warmup=5):
         plx.parallax_decode_fwd_ex(x["q"], x["r"], x["k"], x["v"], x["seqlens"], out, cfg.scale, ws, 0, st or stream)
     for i in range(warmup):
         step(i)
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for i in range(steps):
-        step(i)
-    e1.record(stream)
-    torch.cuda.synchronize()
-    us = e0.elapsed_time(e1) / steps * 1e3
+    t = BlockTimer(stream, sampler).run(step, steps)
+    us = t["ms_per_step"] * 1e3
     peak, _ = measured_peaks()
-    return {"us_per_call": round(us, 2), "us_per_call_graph_replay": round(graph_replay_us(step, nsets), 2),
-            "kv_read_TBps": round(kv_bytes / us / 1e6, 4),
-            "frac_of_measured_copy_bw": round(kv_bytes / us / 1e3 / peak, 4),
-            "frac_of_8TBps_nominal": round(kv_bytes / us / 1e3 / 8000.0, 4), "kv_bytes": kv_bytes}
+    traffic, traffic_src = ncu_traffic(name)
+    res = {"us_per_call": round(us, 2), "us_per_call_graph_replay": round(graph_replay_us(step, nsets), 2),
+           "kv_read_TBps": round(kv_bytes / us / 1e6, 4),
+           "frac_of_measured_copy_bw": round(kv_bytes / us / 1e3 / peak, 4),
+           "frac_of_8TBps_nominal": round(kv_bytes / us / 1e3 / 8000.0, 4), "kv_bytes": kv_bytes,
+           "traffic": traffic, "traffic_source": traffic_src, "clocks": t["clocks"], **timing_note(t)}
+    if read_peak:
+        res["frac_of_read_probe"] = round(kv_bytes / us / 1e3 / read_peak, 4)
+    return res
+
+
+def quick_tensor_workload(name, local_rank=0):
+    """Short run of a tensor-core workload (multi-token forward or backward) for the default line: value,
+    roofline fraction against the sustained bf16 peak, clocks."""
+    ns = argparse.Namespace(workload=name, steps=5, warmup=3, batch=0, kv_sets=0, plain_bf16_p=False,
+                            no_cpu_baseline=True, cpu_seconds=0.0)
+    runner = run_prefill if name in wl.PREFILL_CONFIGS else run_backward
+    r = runner(ns, 0, 1, local_rank)
+    torch.cuda.empty_cache()
+    return {"metric": r["metric"], "value": r["value"], "unit": r["unit"], "ms_per_step": r["ms_per_step"],
+            "roofline_frac_of_sustained_bf16": r["roofline"]["frac"], "roofline_kernel": r["roofline"]["kernel"],
+            "workload": r["config"]["workload"], "clocks": r["clocks"], **r["timing"]}
+
+
+def single_thread_oracle_c2():
+    """The fp64 oracle on the whole C2 call with ONE thread (seconds per call)."""
+    from oracle import parallax_oracle as po
+    po.build()
+    cfg = wl.CONFIGS["C2"]
+    x = wl.make_inputs(cfg, "cuda" if torch.cuda.is_available() else "cpu")
+    bits = {n: wl.bf16_bits(x[n]) for n in ("q", "r", "k", "v")}
+    t0 = time.perf_counter()
+    _, threads = po.decode_bf16(bits["q"], bits["r"], bits["k"], bits["v"], None, cfg.scale, threads=1)
+    secs = time.perf_counter() - t0
+    return {"seconds_per_call": round(secs, 4), "value": round(cfg.kv_bytes() / secs / 1e12, 8), "unit": UNIT,
+            "cores": threads, "sample": "the whole C2 call (64 (sequence, kv-head) streams of 4096 keys), one thread"}
 
 
 def run_prefill(args, rank, world, local_rank):
@@ -461,27 +607,12 @@ def run_prefill(args, rank, world, local_rank):
         x = sets[i % nsets]
         plx.parallax_prefill_fwd_ex(x["q"], x["r"], x["k"], x["v"], None, out, cfg.scale, ws, 0, status, stream, prec)
 
-    def barrier():
-        if world > 1:
-            torch.distributed.barrier()
-        torch.cuda.synchronize()
-
-    def timed(fn, steps):
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        sampler.active.set()
-        e0.record(stream)
-        for i in range(steps):
-            fn(i)
-        e1.record(stream)
-        barrier()
-        sampler.active.clear()
-        return max_over_ranks(e0.elapsed_time(e1), world, dev)
-
     sampler = ClockSampler(local_rank)
+    timer = BlockTimer(stream, sampler, world, dev)
     for i in range(args.warmup):
         step(i)
-    ms = timed(step, args.steps) / args.steps
+    t_call = timer.run(step, args.steps)
+    ms = t_call["ms_per_step"]
     assert int(status.item()) == 0, "device-side wait timed out"
     value = flops * world / (ms * 1e-3) / 1e12
 
@@ -501,8 +632,9 @@ def run_prefill(args, rank, world, local_rank):
     e2e_steps = max(5, args.steps // 10)
     for i in range(2):
         e2e_step(i)
-    ms_e2e = timed(e2e_step, e2e_steps) / e2e_steps
-    clocks = sampler.summary()
+    ms_e2e = timer.run(e2e_step, e2e_steps)["ms_per_step"]
+    clocks = t_call["clocks"]
+    sampler.close()
 
     peaks = json.loads((ROOT / "MEASURED_PEAKS.json").read_text()) if (ROOT / "MEASURED_PEAKS.json").exists() else None
     peak = float(peaks["bf16_tflops_sustained"]) if peaks else 1400.0
@@ -526,11 +658,12 @@ def run_prefill(args, rank, world, local_rank):
                      "executed_tflops_incl_residual_mmas": round(achieved * mma_factor, 1),
                      "p_precision": "bf16" if args.plain_bf16_p else "bf16+residual",
                      "algorithmic_flops_per_launch": flops,
-                     "traffic": None if args.batch else NCU_TRAFFIC_BYTES.get(cfg.name)},
+                     "traffic": None if args.batch else ncu_traffic(cfg.name)[0],
+                     "traffic_source": None if args.batch else ncu_traffic(cfg.name)[1]},
         "e2e": {"value": round(flops * world / (ms_e2e * 1e-3) / 1e12, 2), "unit": "TFLOP/s",
                 "ms_per_step": round(ms_e2e, 4), "h2d_bytes_per_step": 2 * n_q, "d2h_bytes_per_step": n_q,
                 "note": "q and r copied from pinned host memory and the output copied back every step"},
-        "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+        "gpu_launches": launches_per_step * args.steps * t_call["blocks"], "clocks": clocks, "timing": timing_note(t_call),
     }
     if launches_per_step > 1:
         result["config"]["split_kv"] = ("the row tiles alone leave SMs idle: the library divides each tile's keys among "
@@ -598,27 +731,12 @@ def run_backward(args, rank, world, local_rank):
         plx.parallax_prefill_bwd(x["q"], x["r"], x["k"], x["v"], x["dout"] if dout is None else dout, x["out"], x["lse"],
                                  x["tbar"], x["vbar"], None, dq, dr, dk, dv, cfg.scale, ws, status, stream)
 
-    def barrier():
-        if world > 1:
-            torch.distributed.barrier()
-        torch.cuda.synchronize()
-
-    def timed(fn, steps):
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        sampler.active.set()
-        e0.record(stream)
-        for i in range(steps):
-            fn(i)
-        e1.record(stream)
-        barrier()
-        sampler.active.clear()
-        return max_over_ranks(e0.elapsed_time(e1), world, dev)
-
     sampler = ClockSampler(local_rank)
+    timer = BlockTimer(stream, sampler, world, dev)
     for i in range(args.warmup):
         step(i)
-    ms = timed(step, args.steps) / args.steps
+    t_call = timer.run(step, args.steps)
+    ms = t_call["ms_per_step"]
     assert int(status.item()) == 0, "device-side wait timed out"
     value = flops * world / (ms * 1e-3) / 1e12
 
@@ -636,8 +754,9 @@ def run_backward(args, rank, world, local_rank):
     e2e_steps = max(3, args.steps // 10)
     for i in range(2):
         e2e_step(i)
-    ms_e2e = timed(e2e_step, e2e_steps) / e2e_steps
-    clocks = sampler.summary()
+    ms_e2e = timer.run(e2e_step, e2e_steps)["ms_per_step"]
+    clocks = t_call["clocks"]
+    sampler.close()
 
     peaks = json.loads((ROOT / "MEASURED_PEAKS.json").read_text()) if (ROOT / "MEASURED_PEAKS.json").exists() else None
     peak = float(peaks["bf16_tflops_sustained"]) if peaks else 1400.0
@@ -661,11 +780,12 @@ def run_backward(args, rank, world, local_rank):
                      "unit": "TFLOP/s", "frac": round(achieved / peak, 4), "frac_of_burst_peak": round(achieved / burst, 4),
                      "executed_tflops_incl_recomputed_scores": round(achieved * 22.0 / 16.0, 1),
                      "algorithmic_flops_per_launch": flops,
-                     "traffic": None if args.batch else NCU_TRAFFIC_BYTES.get(cfg.name)},
+                     "traffic": None if args.batch else ncu_traffic(cfg.name)[0],
+                     "traffic_source": None if args.batch else ncu_traffic(cfg.name)[1]},
         "e2e": {"value": round(flops * world / (ms_e2e * 1e-3) / 1e12, 2), "unit": "TFLOP/s",
                 "ms_per_step": round(ms_e2e, 4), "h2d_bytes_per_step": n_q, "d2h_bytes_per_step": 2 * n_q + 2 * n_kv,
                 "note": "dO copied from pinned host memory and dq, dr, dk, dv copied back every step"},
-        "gpu_launches": 3 * args.steps, "clocks": clocks,
+        "gpu_launches": 3 * args.steps * t_call["blocks"], "clocks": clocks, "timing": timing_note(t_call),
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import parallax_oracle as po
@@ -748,6 +868,116 @@ def run_grid(args):
                 del ks, vs
 
 
+def run_sharded(args, rank, world, local_rank):
+    """--shard-keys: ONE batch whose keys are divided among the ranks (strong scaling).  Every rank holds
+    T/world keys of every sequence and, per step: split kernel on its slice -> all-gather of the ~1 KB
+    records (NCCL; skipped on one rank) -> combine kernel over all ranks' records.  value = the whole
+    context's K/V bytes / the slowest rank's time."""
+    from paper_2605_29157_b200 import binding as plx
+    from paper_2605_29157_b200 import sequence_parallel as sp
+
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    cfg = wl.CONFIGS[args.workload]
+    if cfg.ragged is not None:
+        raise SystemExit("--shard-keys needs a uniform-context workload (C4 is the one it is meant for)")
+    if cfg.T_max % (world * 64):
+        raise SystemExit(f"--shard-keys: context {cfg.T_max} is not a multiple of 64 * {world} ranks")
+    T_shard = cfg.T_max // world
+    shard_cfg = wl.scaled(cfg, T_max=T_shard)
+    set_bytes = cfg.B * cfg.Hkv * T_shard * cfg.D * 4
+    nsets = args.kv_sets or min(16, max(2, -(-(1 << 30) // set_bytes)))
+    # q, r are replicated (same seed on every rank); each rank draws its own slice of the caches
+    qr = wl.make_inputs(wl.scaled(shard_cfg, T_max=64), dev)
+    sets = [wl.make_inputs(wl.scaled(shard_cfg, seed=rank_seed(cfg.seed, rank) + 17 * i), dev, kv_only=True)
+            for i in range(nsets)]
+    chunk, ns = sp.plan_shard(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, T_shard, dev)
+    stride = plx.parallax_partial_stride(cfg.D)
+    partials = torch.empty(cfg.B, cfg.Hq, ns, stride, dtype=torch.float32, device=dev)
+    out = torch.empty(cfg.B, cfg.Hq, cfg.D, dtype=torch.bfloat16, device=dev)
+    stream = torch.cuda.current_stream()
+    kv_bytes = cfg.kv_bytes()
+
+    def step(i):
+        x = sets[i % nsets]
+        sp.decode_sequence_sharded(qr["q"], qr["r"], x["k"], x["v"], None, out, cfg.scale, chunk, None, partials)
+
+    def local_only(i):
+        x = sets[i % nsets]
+        plx.parallax_decode_splitkv_partial(qr["q"], qr["r"], x["k"], x["v"], None, partials, cfg.scale, chunk, ns,
+                                            None, stream)
+    sampler = ClockSampler(local_rank)
+    timer = BlockTimer(stream, sampler, world, dev)
+    for i in range(args.warmup):
+        step(i)
+    t_call = timer.run(step, args.steps)
+    for i in range(3):
+        local_only(i)
+    t_kernel = timer.run(local_only, args.steps)
+    peak, peak_src = measured_peaks()
+    achieved = kv_bytes / world / (t_kernel["ms_per_step"] * 1e-3) / 1e9
+    ms = t_call["ms_per_step"]
+    result = {
+        "metric": METRIC, "value": round(kv_bytes / (ms * 1e-3) / 1e12, 4), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms, 6), "us_per_call": round(ms * 1e3, 2),
+        "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{cfg.name}: {cfg.note}; B={cfg.B} Hq={cfg.Hq} Hkv={cfg.Hkv} D={cfg.D} context={cfg.T_max} "
+                               f"uniform, keys sharded over {world} rank(s) ({T_shard} keys per sequence and rank)",
+                   "B": cfg.B, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D, "T_max": cfg.T_max, "T_shard": T_shard,
+                   "chunk_len": chunk, "num_splits_per_rank": ns,
+                   "l2_policy": f"{nsets} cache slices per rank used round-robin ({nsets * set_bytes / 2**30:.3f} GiB vs 0.123 GiB L2)",
+                   "parallelism": f"keys of every sequence sharded over {world} rank(s); per step: split kernel -> "
+                                  "all-gather of the partial records -> combine kernel on every rank",
+                   "collective_bytes_per_rank": cfg.B * cfg.Hq * ns * stride * 4},
+        "roofline": {"bound": "hbm", "kernel": "plx_decode_kernel (one rank's slice)", "achieved": round(achieved, 1),
+                     "peak": peak, "peak_source": f"{peak_src} copy bandwidth (read + write)", "unit": "GB/s",
+                     "frac": round(achieved / peak, 4), "us_per_launch": round(t_kernel["ms_per_step"] * 1e3, 2),
+                     "algorithmic_bytes_per_launch": kv_bytes // world, "traffic": None},
+        "e2e": None, "gpu_launches": 2 * args.steps * t_call["blocks"], "clocks": t_call["clocks"],
+        "timing": timing_note(t_call),
+    }
+    sampler.close()
+    return result
+
+
+def run_launcher_selftest(args, rank, world):
+    """Rehearsal of the multi-rank plumbing on CPU ranks (gloo): the same launcher, rendezvous, per-rank
+    seeding, max-over-ranks reduction, record gather and one-line report as a GPU run, with NO kernel and
+    therefore no measurement (value is null).  Exists so that the launcher can be tested without GPUs."""
+    from paper_2605_29157_b200 import sequence_parallel as sp
+    cfg = wl.scaled(wl.CONFIGS["C1"], seed=rank_seed(0, rank))
+    x = wl.make_inputs(cfg, "cpu")
+    digest = float(x["k"].float().abs().sum())
+    digests = [None] * world
+    torch.distributed.all_gather_object(digests, digest)
+    ms = max_over_ranks(1.0 + rank, world, "cpu")            # stand-in times: rank r "took" 1 + r ms
+    gathered_ok = None
+    if args.shard_keys:                                        # the exchange step on CPU tensors
+        rec = torch.full((2, 4, 3, 20), float(rank))
+        g = sp.gather_partials(rec)
+        gathered_ok = bool(tuple(g.shape) == (world, 2, 4, 3, 20) and all(float(g[w].mean()) == w for w in range(world)))
+    return {"metric": METRIC, "value": None, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "strong" if args.shard_keys else "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "gpu_launches": 0,
+            "selftest": "launcher rehearsal on CPU ranks (gloo): no kernel ran, nothing here is a measurement",
+            "distinct_rank_inputs": len(set(digests)) == world, "stand_in_ms_max_over_ranks": ms,
+            "gathered_layout_ok": gathered_ok, "config": {"workload": "none (launcher rehearsal)"}}
+
+
+def launch_ranks(args, argv):
+    """`--gpus N` outside a torchrun environment: start N ranks of this script (one process per GPU) under
+    torch.distributed.run and pass their exit code on.  Never runs fewer ranks than asked for."""
+    n = args.gpus
+    if not args.launcher_selftest:
+        have = torch.cuda.device_count()
+        if have < n:
+            print(f"bench.py: --gpus {n} asked for, {have} CUDA device(s) visible; refusing to run fewer ranks", file=sys.stderr)
+            return 2
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), str(Path(__file__).resolve())] + argv
+    return subprocess.call(cmd)
+
+
 def run_reference(args):
     """The oracle, as it stands, on the host cores: each step is a bounded sample of the workload."""
     if args.workload in wl.PREFILL_CONFIGS or args.workload in wl.BACKWARD_CONFIGS:
@@ -783,14 +1013,19 @@ def run_reference(args):
     }
 
 
-def main():
+def main(argv=None):
+    argv = list(sys.argv[1:] if argv is None else argv)
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--workload", default="C3", choices=sorted(wl.CONFIGS) + sorted(wl.PREFILL_CONFIGS) + sorted(wl.BACKWARD_CONFIGS))
+    ap.add_argument("--workload", default=None, choices=sorted(wl.CONFIGS) + sorted(wl.PREFILL_CONFIGS) + sorted(wl.BACKWARD_CONFIGS),
+                    help="default C3 (C4 with --shard-keys)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--fp8-kv", action="store_true", help="decode workloads over an e4m3 KV cache (D = 128)")
+    ap.add_argument("--shard-keys", action="store_true",
+                    help="strong scaling: the keys of every sequence are divided among the ranks (split kernel, "
+                         "all-gather of the partial records, combine)")
+    ap.add_argument("--fp8-kv", action="store_true", help="decode workloads over an e4m3 KV cache")
     ap.add_argument("--splits", type=int, default=0, help="force the split count (0 = library plan)")
     ap.add_argument("--kv-sets", type=int, default=0, help="number of KV cache sets rotated between steps")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (profiling captures on a smaller case)")
@@ -801,12 +1036,20 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--grid", action="store_true", help="decode sweep over the paper's batch x context grid (one JSON line per cell)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-read-probe", action="store_true", help="skip the read-only streaming probe (profiling captures)")
     ap.add_argument("--no-other-configs", dest="all_configs", action="store_false",
                     help="skip the short runs of the other decode configurations that ride along in the default line")
-    args = ap.parse_args()
+    ap.add_argument("--launcher-selftest", action="store_true",
+                    help="rehearse the multi-rank plumbing on CPU ranks (gloo): no kernel, no measurement")
+    args = ap.parse_args(argv)
     if args.warmup < 3:
         args.warmup = 3
+    if args.workload is None:
+        args.workload = "C4" if args.shard_keys else "C3"
+    if args.gpus < 1:
+        ap.error("--gpus must be >= 1")
 
+    in_torchrun = "WORLD_SIZE" in os.environ
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -814,23 +1057,43 @@ def main():
     if args.impl == "reference":
         if rank == 0:
             print(json.dumps(run_reference(args)), flush=True)
-        return
+        return 0
     if args.grid:
         if rank == 0:
             run_grid(args)
-        return
+        return 0
+    if not in_torchrun and args.gpus > 1:
+        return launch_ranks(args, argv)
+    if in_torchrun and world != args.gpus:
+        print(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s)", file=sys.stderr)
+        return 2
 
-    if world > 1:
-        torch.cuda.set_device(local_rank)
-        torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    runner = run_prefill if args.workload in wl.PREFILL_CONFIGS else run_backward if args.workload in wl.BACKWARD_CONFIGS else run_ours
-    result = runner(args, rank, world, local_rank)
+    if args.launcher_selftest:
+        if world > 1:
+            torch.distributed.init_process_group("gloo")
+        result = run_launcher_selftest(args, rank, world) if world > 1 else {"selftest": "one rank: nothing to rehearse", "n_gpus": 1}
+    else:
+        if not torch.cuda.is_available() or torch.cuda.device_count() <= local_rank:
+            print("bench.py: no CUDA device for this rank (the CUDA library is the only implementation)", file=sys.stderr)
+            return 2
+        if world > 1:
+            torch.cuda.set_device(local_rank)
+            torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        if args.shard_keys:
+            if args.workload not in wl.CONFIGS:
+                ap.error("--shard-keys applies to the decode workloads")
+            runner = run_sharded
+        else:
+            runner = (run_prefill if args.workload in wl.PREFILL_CONFIGS else
+                      run_backward if args.workload in wl.BACKWARD_CONFIGS else run_ours)
+        result = runner(args, rank, world, local_rank)
     if rank == 0:
         print(json.dumps(result), flush=True)
     if world > 1:
         torch.distributed.barrier()
         torch.distributed.destroy_process_group()
+    return 0
 
 
 if __name__ == "__main__":
-    main()
+    sys.exit(main())

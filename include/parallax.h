@@ -62,6 +62,7 @@ extern "C" {
 #define PLX_ERR_CUDA (-7)
 #define PLX_ERR_DEVICE_TIMEOUT (-8)
 #define PLX_ERR_STATIC_SCRATCH (-9)
+#define PLX_ERR_DEVICE_CHECK (-10) /* debug build only (PLX_DEBUG_CHECKS): a kernel refused an out-of-range index */
 
 #define PLX_OUT_BF16 0
 #define PLX_OUT_F32 1
@@ -525,6 +526,28 @@ int parallax_decode_step(const void* q_raw, const void* r_raw, const void* k_raw
 int parallax_decode_fwd_static(const void* q, const void* r, const void* k_cache, const void* v_cache,
                                const int32_t* seqlens, void* out, int B, int Hq, int Hkv, int D,
                                int T_max, float scale, int out_dtype, int num_splits, void* stream);
+
+/*
+ * Read-only streaming probe (a measurement aid; the paper has no counterpart).  The decode forward
+ * only reads the K/V stream (Sec. 3.3: the KV stream is the cost), so its bandwidth ceiling is the
+ * rate at which a kernel can read HBM and keep nothing, not the rate of a copy.  This call reads
+ * `bytes` bytes at `src` (device, 16-byte aligned; bytes a multiple of 8192) exactly once:
+ *   mode PLX_PROBE_VECTOR_LOADS  16-byte L1-bypassing loads, eight independent loads per thread;
+ *   mode PLX_PROBE_BULK_COPIES   bulk asynchronous copies of 8 KiB into warp-private three-slot
+ *                                shared-memory rings, two CTAs per SM (the staging geometry of
+ *                                the decode kernel at D = 128 with the arithmetic removed).
+ * `ctas` = number of CTAs, each reading one contiguous range (0 = eight per SM for vector loads,
+ * two per SM for bulk copies).  `sink` (device, 16-byte aligned, PLX_PROBE_SINK_BYTES bytes) receives
+ * one 16-byte store per CTA (per warp in bulk mode) so that the loads are live; its contents mean
+ * nothing.  `status` (device int32, may be NULL) receives PLX_ERR_DEVICE_TIMEOUT if a bounded wait of
+ * the bulk mode runs out.  One launch on `stream`; nothing is allocated.  Time it with events:
+ * bandwidth = bytes / elapsed.
+ */
+#define PLX_PROBE_VECTOR_LOADS 0
+#define PLX_PROBE_BULK_COPIES 1
+#define PLX_PROBE_SINK_BYTES 65536
+int parallax_read_probe(const void* src, size_t bytes, void* sink, int mode, int ctas, int32_t* status,
+                        void* stream);
 
 #ifdef __cplusplus
 }

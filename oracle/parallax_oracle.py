@@ -20,7 +20,8 @@ Contents
                             right-hand side; Sigma_KV as defined under
                             Eq. "parameterized_lla")
     - ``expanded_form``     Eq. "parallax_expand" (Sec. 3.3)
-    - ``streaming_alg1``    Algorithm 1, tile by tile, with its final line
+    - ``streaming_fold``    the one-pass tile walk of Sec. 3.3 (Algorithm 1) as a running fold of
+                            per-tile states, with its final line
     - ``partial_state`` / ``merge_partials``  the unnormalised per-split state
                             (m, d1, d2, O1, O2) and the log-sum-exp merge of
                             App. "Kernel Optimization Details", item 3
@@ -231,28 +232,6 @@ def expanded_form(q, r, K, V, scale):
     return (p @ V) * (1.0 + p @ t) - (p * t) @ V
 
 
-def streaming_alg1(q, r, K, V, scale, Bc):
-    """Algorithm 1 (Sec. 3.3) for one query row, column tiles of Bc keys.  The paper writes
-    exp2 with log2(e) folded into s; natural exp with the plain scale is the same quantity."""
-    L, Dv = K.shape[0], V.shape[1]
-    m_r, d1, d2 = -np.inf, 0.0, 0.0
-    O1, O2 = np.zeros(Dv), np.zeros(Dv)
-    for c0 in range(0, L, Bc):
-        Kc, Vc = K[c0:c0 + Bc], V[c0:c0 + Bc]
-        S1 = (Kc @ q) * scale
-        m = max(m_r, S1.max())
-        alpha = np.exp(m_r - m)
-        P1 = np.exp(S1 - m)
-        m_r = m
-        S2 = Kc @ r
-        P2 = P1 * S2
-        d1 = alpha * d1 + P1.sum()
-        d2 = alpha * d2 + P2.sum()
-        O1 = alpha * O1 + P1 @ Vc
-        O2 = alpha * O2 + P2 @ Vc
-    return O1 / d1 * (1.0 + d2 / d1) - O2 / d1
-
-
 def partial_state(q, r, K, V, scale, k0, k1):
     """Unnormalised state (m, d1, d2, O1, O2) of the key range [k0, k1), relative to its own
     maximum logit m (natural-log units); an empty range gives (-inf, 0, 0, 0, 0)
@@ -285,6 +264,23 @@ def merge_partials(states):
         d2 += a * a2
         O1 += a * B1
         O2 += a * B2
+    return O1 / d1 * (1.0 + d2 / d1) - O2 / d1
+
+
+def streaming_fold(q, r, K, V, scale, Bc):
+    """The single-pass computation of Sec. 3.3 (Algorithm 1) for one query row, stated as a running
+    fold: the context is walked once in tiles of Bc keys; each tile's unnormalised state is taken
+    relative to the tile's own maximum logit and absorbed into the running state, whichever of the two
+    has the smaller reference being rescaled to the larger one.  Both branches (softmax sums and
+    probe-weighted sums) share the one reference exponent, which only the softmax logits determine.
+    Natural exp with the plain scale; the paper's exp2 with log2(e) folded into s is the same quantity."""
+    run = (-np.inf, 0.0, 0.0, np.zeros(V.shape[1]), np.zeros(V.shape[1]))
+    for lo in range(0, K.shape[0], Bc):
+        tile = partial_state(q, r, K, V, scale, lo, min(lo + Bc, K.shape[0]))
+        ref = max(run[0], tile[0])
+        keep, take = np.exp(run[0] - ref), np.exp(tile[0] - ref)
+        run = (ref,) + tuple(keep * a + take * b for a, b in zip(run[1:], tile[1:]))
+    _, d1, d2, O1, O2 = run
     return O1 / d1 * (1.0 + d2 / d1) - O2 / d1
 
 

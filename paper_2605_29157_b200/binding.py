@@ -8,6 +8,7 @@ library and raises if it has not been built: there is no fallback.
 from __future__ import annotations
 
 import ctypes
+import os
 from pathlib import Path
 from typing import Optional
 
@@ -23,6 +24,10 @@ PLX_ERR_NEED_LAYOUT = -6
 PLX_ERR_CUDA = -7
 PLX_ERR_DEVICE_TIMEOUT = -8
 PLX_ERR_STATIC_SCRATCH = -9
+PLX_ERR_DEVICE_CHECK = -10
+PLX_PROBE_VECTOR_LOADS = 0
+PLX_PROBE_BULK_COPIES = 1
+PLX_PROBE_SINK_BYTES = 65536
 PLX_STATIC_SCRATCH_BYTES = 8 * 1024 * 1024
 PLX_OUT_BF16 = 0
 PLX_OUT_F32 = 1
@@ -30,7 +35,9 @@ PLX_P_BF16_RESIDUAL = 0
 PLX_P_BF16 = 1
 PLX_MAX_SPLITS = 1024
 
-LIB_PATH = Path(__file__).resolve().parent / "libparallax.so"
+# PARALLAX_LIBRARY selects another build of the same library (the index-checking debug build,
+# `python -m paper_2605_29157_b200.build --debug-checks`); the default is the optimised in-tree build.
+LIB_PATH = Path(os.environ.get("PARALLAX_LIBRARY") or Path(__file__).resolve().parent / "libparallax.so")
 
 EXPORTS = (
     "parallax_version", "parallax_status_string", "parallax_partial_stride",
@@ -44,7 +51,9 @@ EXPORTS = (
     "parallax_decode_step", "parallax_decode_fwd_fp8_per_head", "parallax_decode_fwd_paged_fp8_per_head",
     "parallax_decode_fwd_multi", "parallax_prefill_workspace_bytes", "parallax_prefill_fwd_ex",
     "parallax_prefill_fwd_paged_ex", "parallax_decode_fwd_multi_paged", "parallax_decode_fwd_args",
+    "parallax_read_probe",
 )
+TEST_HOOK_EXPORTS = ("plx_test_bounded_wait",)
 
 
 class ParallaxError(RuntimeError):
@@ -94,6 +103,8 @@ def _load() -> ctypes.CDLL:
         "parallax_decode_step": (i32, [vp] * 13 + [i32, i32, i32, i32, i32, f32, f32, i32, f32, i32, vp, sz, i32, vp]),
         "parallax_decode_fwd_paged": (i32, [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, f32, i32,
                                             vp, sz, i32, vp]),
+        "parallax_read_probe": (i32, [vp, sz, vp, i32, i32, vp, vp]),
+        "plx_test_bounded_wait": (i32, [vp, ctypes.c_uint32, vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -587,3 +598,18 @@ def parallax_decode_prepare(q_raw, r_raw, k_raw, v_raw, q_weight, r_weight, k_we
                                         _ptr(r_weight), _ptr(k_weight), _ptr(seqlens), _ptr(q_out), _ptr(r_out),
                                         _ptr(k_cache), _ptr(v_cache), B, Hq, Hkv, D, T_max, float(eps),
                                         float(rope_theta), int(bool(rope_on_r)), _stream(stream)))
+
+
+def parallax_read_probe(src, sink, mode=PLX_PROBE_VECTOR_LOADS, ctas=0, status=None, stream=None, nbytes=None):
+    """Reads `nbytes` (default: all) of the device tensor `src` once; `sink` is a device tensor of at
+    least PLX_PROBE_SINK_BYTES bytes."""
+    _require(src, sink)
+    total = src.numel() * src.element_size() if nbytes is None else int(nbytes)
+    if sink.numel() * sink.element_size() < PLX_PROBE_SINK_BYTES:
+        raise ParallaxError(PLX_ERR_BAD_SHAPE)
+    _check(_lib.parallax_read_probe(_ptr(src), total, _ptr(sink), mode, ctas, _ptr(status), _stream(stream)))
+
+
+def plx_test_bounded_wait(status, attempts, polls_done=None, stream=None):
+    """Test hook: one warp polls a barrier nothing arrives on `attempts` times, then sets `status`."""
+    _check(_lib.plx_test_bounded_wait(_ptr(status), attempts, _ptr(polls_done), _stream(stream)))

@@ -785,6 +785,7 @@ extern "C" int parallax_prefill_bwd(const void* q, const void* r, const void* k_
     float4* stats = static_cast<float4*>(workspace);
     const __nv_bfloat16* g = static_cast<const __nv_bfloat16*>(dout);
 
+    PlxNvtxRange nvtx_range("plx_prefill_bwd(prep, row pass, column pass)");
     // the padding records past the last row are read by the column pass (and masked): keep them finite
     if (cudaMemsetAsync(stats + q_rows, 0, BN * sizeof(float4), st) != cudaSuccess) return PLX_ERR_CUDA;
     const unsigned prep_grid = static_cast<unsigned>((q_rows + 7) / 8);

@@ -112,7 +112,15 @@ struct KernelParams {
     // host only: launch as a programmatic dependent of the previous kernel in the stream (the kernel's
     // first instruction waits for that kernel's results; see parallax_decode_step)
     int dependent_launch = 0;
+    // What the host knows about the buffers, for the index checks of the debug build (PLX_DEBUG_CHECKS):
+    // rows each K/V tensor map covers, and the number of records `partials` has room for.
+    long long kv_rows = 0;
+    long long partial_records = 0;
 };
+
+#ifndef PLX_DEBUG_CHECKS
+#define PLX_DEBUG_CHECKS 0
+#endif
 
 // ---------------------------------------------------------------------------
 // Warp-level MMA helpers (the mbarrier / TMA wrappers live in plx_common.cuh)
@@ -406,6 +414,27 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     }
     const int k1 = min(k0 + p.chunk_len, L);
     const int ntiles = (k1 - k0 + kTileKeys - 1) / kTileKeys;
+#if PLX_DEBUG_CHECKS
+    {
+        // Debug build: every index this CTA will form is affine in values known here, so the extremes are
+        // checked once, CTA-uniformly; a violation is reported through the status word and the CTA leaves
+        // without touching the address (page ids, which are data, are checked where they are read).
+        const int hkv_r = hkv / p.kv_div, Hkv_r = p.Hkv / p.kv_div;
+        bool ok = stream_id < p.B * p.Hkv && p.Hq == p.Hkv * G && p.Hkv % p.kv_div == 0 && p.lq >= 1 &&
+                  p.chunk_len % kTileKeys == 0 && static_cast<long long>(p.chunk_len) * p.num_splits >= p.T_max;
+        if (!p.block_table)
+            ok = ok && (static_cast<long long>(b) * Hkv_r + hkv_r) * p.T_max + k1 <= p.kv_rows;
+        else
+            ok = ok && p.page_size > 0 && p.page_size % kTileKeys == 0 && (k1 + p.page_size - 1) / p.page_size <= p.max_pages;
+        if (p.mode != kModeFinal)
+            ok = ok && (static_cast<long long>(b) * p.Hq + hkv * G + (G - 1)) * p.num_splits + split < p.partial_records;
+        if (p.mode == kModeFused) ok = ok && p.counters != nullptr;
+        if (!ok) {
+            if (threadIdx.x == 0 && p.status) atomicExch(p.status, PLX_ERR_DEVICE_CHECK);
+            return;
+        }
+    }
+#endif
     const int n_my = (ntiles - warp + kWarps - 1) / kWarps;  // tiles warp, warp+4, ... (may be 0)
 
     const uint32_t ring = base_addr + warp * NSTAGES * SL::kStageBytes;
@@ -444,6 +473,12 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         if (pg != pg_cur) {
             pg_id_cur = (pg_cur >= 0 && pg == pg_cur + 1) ? pg_id_next : __ldg(table + pg);
             pg_cur = pg;
+#if PLX_DEBUG_CHECKS
+            if (pg_id_cur < 0 || (static_cast<long long>(pg_id_cur) * Hkv_real + hkv_real + 1) * p.page_size > p.kv_rows) {
+                if (p.status) atomicExch(p.status, PLX_ERR_DEVICE_CHECK);  // a page id outside the pool: not followed
+                pg_id_cur = 0;
+            }
+#endif
             if (pg + 1 < p.max_pages) pg_id_next = __ldg(table + pg + 1);
         }
         return (pg_id_cur * Hkv_real + hkv_real) * p.page_size + (key - pg * p.page_size);
@@ -1074,6 +1109,8 @@ int launch_main(const CUtensorMap& tmK, const CUtensorMap& tmV, const KernelPara
 {
     using SL = SmemLayout<D, NSTAGES, FP8>;
     auto kernel = plx_decode_kernel<D, G, NSTAGES, CTAS, FP8>;
+    PlxNvtxRange nvtx_range(kp.mode == kModeFinal ? "plx_decode_main(final)" : kp.mode == kModeFused ? "plx_decode_main(fused merge)"
+                                                                                                    : "plx_decode_main(partial)");
     static bool configured[64] = {false};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return PLX_ERR_CUDA;
@@ -1164,6 +1201,7 @@ int launch_combine(const float* partials, const int32_t* split_counts, const int
                    int T_max, void* out, int B, int Hq, int D, int num_splits, int out_dtype, cudaStream_t stream,
                    int num_groups = 1, bool dependent_launch = false)
 {
+    PlxNvtxRange nvtx_range("plx_decode_combine");
     const size_t group_stride = static_cast<size_t>(B) * Hq * num_splits * (2 * D + 4);
     const unsigned rows = static_cast<unsigned>(B * Hq);
     if (dependent_launch) {
@@ -1276,6 +1314,7 @@ const char* parallax_status_string(int status)
         case PLX_ERR_CUDA: return "CUDA runtime or driver call failed";
         case PLX_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
         case PLX_ERR_STATIC_SCRATCH: return "requested splits need more scratch than the built-in static array holds";
+        case PLX_ERR_DEVICE_CHECK: return "debug build: a kernel refused an out-of-range index";
         default: return "unknown status";
     }
 }
@@ -1316,6 +1355,8 @@ int parallax_decode_splitkv_partial(const void* q, const void* r, const void* k_
     KernelParams kp{static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(r), seqlens, nullptr,
                     partials, status, nullptr, nullptr, 0, 0, B, Hq, Hkv, T_max, chunk_len, num_splits, scale * kLog2e, PLX_OUT_F32,
                     kModePartialWriteEmpty};
+    kp.kv_rows = static_cast<long long>(rows);
+    kp.partial_records = static_cast<long long>(B) * Hq * num_splits;
     const int g = apply_group(&kp, Hq, Hkv);
     return dispatch_main(D, g, tmK, tmV, kp, static_cast<cudaStream_t>(stream));
 }
@@ -1398,6 +1439,9 @@ static int decode_fwd_impl(const void* q, const void* r, const void* k_cache, co
     }
     kp.dependent_launch = dependent_launch ? 1 : 0;
     kp.lq = lq;
+    kp.kv_rows = static_cast<long long>(rows);
+    if (partials)
+        kp.partial_records = static_cast<long long>((workspace_bytes - fixed_bytes(B, Hq, D)) / ((2 * D + 4) * sizeof(float)));
     const int g = apply_group(&kp, Hq, Hkv);
     return dispatch_main(D, g, tmK, tmV, kp, st, fp8);
 }
@@ -1715,6 +1759,12 @@ int parallax_decode_fwd_host(const void* q_host, const void* r_host, const void*
     } else if ((rc = check_inputs(q_dev, r_dev, k_cache, v_cache, B, Hq, Hkv, D, T_max)) != PLX_OK) {
         return rc;
     }
+    if (num_splits < 0 || num_splits > PLX_MAX_SPLITS) return PLX_ERR_BAD_SHAPE;
+    if (num_splits > 1 && !big_group) {  // a forced split count needs its records' room (a planned one adapts)
+        const int chunk = static_cast<int>(align_up((T_max + num_splits - 1) / num_splits, kChunkGranule));
+        const int ns_eff = (T_max + chunk - 1) / chunk;
+        if (ns_eff > 1 && workspace_bytes < fixed_bytes(B, Hq, D) + partial_bytes(B, Hq, D, ns_eff)) return PLX_ERR_WORKSPACE;
+    }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (in_direct) {
         const size_t n16 = n * 2 / 16;
@@ -1756,12 +1806,14 @@ int parallax_workspace_status(const void* workspace, int32_t* status_host, void*
 // Allocation-free variant of the decode forward.
 //
 // Some callers cannot hand the library a workspace because they cannot allocate
-// device memory at the point where they decode: code running inside a CUDA-graph
-// capture or another region where cudaMalloc is illegal, plug-ins that live
-// inside a host framework's memory pool and are forbidden to allocate behind its
-// back, and real-time loops that must not hit the allocator's locks.  For them
-// the split-KV partial records live in the fixed array below, which every device
-// that loads this library carries until the process exits.
+// device memory at the point where they decode: code running in a region where
+// cudaMalloc is not allowed, plug-ins that live inside a host framework's memory
+// pool and are forbidden to allocate behind its back, and real-time loops that
+// must not hit the allocator's locks.  For them the split-KV partial records live
+// in the fixed array below, which every device that loads this library carries
+// until the process exits.  The first call on a device looks the array's address
+// up, and the first call of a shape (head dimension, group size) on a device sets
+// that kernel's shared-memory attribute: make those calls before any stream capture.
 // ---------------------------------------------------------------------------
 namespace {
 
@@ -1831,6 +1883,8 @@ extern "C" int parallax_decode_fwd_static(const void* q, const void* r, const vo
     KernelParams kp{static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(r), seqlens, out,
                     partials, nullptr, nullptr, nullptr, 0, 0, B, Hq, Hkv, T_max, chunk_len, ns, scale * kLog2e, out_dtype,
                     ns > 1 ? kModePartial : kModeFinal};
+    kp.kv_rows = static_cast<long long>(rows);
+    kp.partial_records = PLX_STATIC_SCRATCH_BYTES / ((2 * D + 4) * sizeof(float));
     const int g = apply_group(&kp, Hq, Hkv);
     if ((rc = dispatch_main(D, g, tmK, tmV, kp, st)) != PLX_OK) return rc;
     if (ns > 1) rc = launch_combine(partials, nullptr, seqlens, chunk_len, T_max, out, B, Hq, D, ns, out_dtype, st);

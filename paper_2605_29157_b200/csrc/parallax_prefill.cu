@@ -733,6 +733,7 @@ static int prefill_impl(const void* q, const void* r, const void* k_cache, const
     const unsigned grid = static_cast<unsigned>(base_ctas * ns);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool res = p_precision == PLX_P_BF16_RESIDUAL;
+    PlxNvtxRange nvtx_range("plx_prefill_fwd");
     if (D == 128) {
         if (res)
             plx_prefill_kernel<true, 128><<<grid, kPrefillThreads, kSmemBytes, st>>>(tmQ, tmR, tmK, tmV, pp);

@@ -14,6 +14,7 @@
 #include <stdint.h>
 
 #include "parallax.h"
+#include "plx_common.cuh"
 
 namespace {
 
@@ -129,6 +130,7 @@ extern "C" int parallax_decode_prepare(const void* q_raw, const void* r_raw, con
                      static_cast<__nv_bfloat16*>(v_cache), B, Hq, Hkv, T_max, eps,
                      log2(static_cast<double>(rope_theta)), rope_on_r};
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    PlxNvtxRange nvtx_range("plx_decode_prepare");
     if (D == 128)
         plx_prepare_kernel<128><<<B, kPrepWarps * 32, 0, st>>>(pp);
     else

@@ -11,7 +11,27 @@
 
 #include "parallax.h"
 
+// NVTX ranges around the library's launches (header-only NVTX v3: no link dependency; without a profiler
+// attached a push/pop pair is two calls through a no-op function pointer).  -DPLX_NVTX=0 removes them.
+#ifndef PLX_NVTX
+#define PLX_NVTX 1
+#endif
+#if PLX_NVTX
+#include <nvtx3/nvToolsExt.h>
+#endif
+
 namespace {
+
+struct PlxNvtxRange {
+#if PLX_NVTX
+    explicit PlxNvtxRange(const char* name) { nvtxRangePushA(name); }
+    ~PlxNvtxRange() { nvtxRangePop(); }
+#else
+    explicit PlxNvtxRange(const char*) {}
+#endif
+    PlxNvtxRange(const PlxNvtxRange&) = delete;
+    PlxNvtxRange& operator=(const PlxNvtxRange&) = delete;
+};
 
 constexpr uint32_t kWaitLimit = 1u << 22;  // mbarrier try_wait attempts before a wait gives up
 
@@ -53,10 +73,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
-// Bounded wait: false if the phase did not complete within kWaitLimit attempts.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+// Bounded wait: false if the phase did not complete within `limit` attempts.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit = kWaitLimit)
 {
-    for (uint32_t i = 0; i < kWaitLimit; ++i)
+    for (uint32_t i = 0; i < limit; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }

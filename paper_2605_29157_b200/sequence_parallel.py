@@ -29,20 +29,34 @@ def gather_partials(partials: torch.Tensor, group: Optional[dist.ProcessGroup] =
     return gathered
 
 
+def plan_shard(B, Hq, Hkv, D, T_shard, device, has_lens=False):
+    """(chunk_len, num_splits) the library plans for one rank's slice."""
+    from . import binding as plx
+    sms = torch.cuda.get_device_properties(device).multi_processor_count
+    chunk_len, _ = plx.parallax_decode_plan(B, Hq, Hkv, D, T_shard, sms, has_lens)
+    return chunk_len, -(-T_shard // chunk_len)
+
+
 def decode_sequence_sharded(q, r, k_shard, v_shard, shard_lens, out, scale, chunk_len: int = 0,
-                            group: Optional[dist.ProcessGroup] = None, stream=None):
+                            group: Optional[dist.ProcessGroup] = None, partials: Optional[torch.Tensor] = None):
     """q, r [B,Hq,D] (replicated), k_shard, v_shard [B,Hkv,T_shard,D] (this rank's slice of every
     sequence), shard_lens int32 [B] valid keys in the slice (None = T_shard).  Every rank ends with the
-    full result in `out`."""
+    full result in `out`.
+
+    All three steps (split kernel, all-gather, combine kernel) are enqueued on torch's CURRENT stream:
+    the collective is ordered against that stream only, so a caller that wants another stream wraps the
+    call in `with torch.cuda.stream(s):`.  `partials` may pass a reusable [B,Hq,num_splits,stride] fp32
+    buffer (steady-state loops allocate nothing then, apart from the gather's output)."""
     from . import binding as plx
     B, Hq, D = q.shape
     T_shard = k_shard.shape[2]
     if chunk_len <= 0:
-        sms = torch.cuda.get_device_properties(q.device).multi_processor_count
-        chunk_len, _ = plx.parallax_decode_plan(B, Hq, k_shard.shape[1], D, T_shard, sms, shard_lens is not None)
+        chunk_len, _ = plan_shard(B, Hq, k_shard.shape[1], D, T_shard, q.device, shard_lens is not None)
     num_splits = -(-T_shard // chunk_len)
     stride = plx.parallax_partial_stride(D)
-    partials = torch.empty(B, Hq, num_splits, stride, dtype=torch.float32, device=q.device)
+    if partials is None:
+        partials = torch.empty(B, Hq, num_splits, stride, dtype=torch.float32, device=q.device)
+    stream = torch.cuda.current_stream(q.device)
     plx.parallax_decode_splitkv_partial(q, r, k_shard, v_shard, shard_lens, partials, scale, chunk_len, num_splits,
                                         None, stream)
     gathered = gather_partials(partials, group)

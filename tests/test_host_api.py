@@ -26,6 +26,11 @@ def test_every_declared_symbol_is_exported(lib):
     for name in declared:
         assert hasattr(lib._lib, name), f"{name} declared in parallax.h but not exported"
     assert declared == set(lib.EXPORTS)
+    hooks = re.sub(r"/\*.*?\*/", "", (ROOT / "include" / "parallax_test_hooks.h").read_text(), flags=re.S)
+    declared_hooks = set(re.findall(r"\b(plx_test_\w+)\s*\(", hooks))
+    assert declared_hooks == set(lib.TEST_HOOK_EXPORTS)
+    for name in declared_hooks:
+        assert hasattr(lib._lib, name), f"{name} declared in parallax_test_hooks.h but not exported"
 
 
 def test_version_and_status_strings(lib):
@@ -186,6 +191,22 @@ def test_serving_variant_entry_points_validate_on_the_host(lib):
     assert paged_prefill(ps=32) == lib.PLX_ERR_BAD_SHAPE      # a 64-key tile must not straddle a page
     assert paged_prefill(prec=9) == lib.PLX_ERR_BAD_SHAPE
     assert paged_prefill(D=96) == lib.PLX_ERR_UNSUPPORTED
+
+
+def test_host_buffer_entry_refuses_a_split_count_without_room_before_staging(lib):
+    """A forced split count whose records do not fit the workspace (or one outside the legal range) is
+    refused by the host-buffer entry before the first copy or launch is enqueued."""
+    L = lib._lib
+    fake = ctypes.c_void_p(0x1000)
+    B, Hq, Hkv, D, T = 2, 4, 2, 128, 8192
+    small = lib.parallax_decode_workspace_bytes(B, Hq, D, 2)
+
+    def host(ns, wsb=small):
+        return L.parallax_decode_fwd_host(fake, fake, fake, fake, None, fake, B, Hq, Hkv, D, T, 0.1, 0, fake, wsb, ns, None)
+
+    assert host(64) == lib.PLX_ERR_WORKSPACE
+    assert host(-1) == lib.PLX_ERR_BAD_SHAPE
+    assert host(lib.PLX_MAX_SPLITS + 1) == lib.PLX_ERR_BAD_SHAPE
 
 
 def test_per_head_scale_and_one_call_step_entry_points_validate_on_the_host(lib):

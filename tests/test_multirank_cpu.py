@@ -1,7 +1,9 @@
 """World-size-2 check of the bench's multi-rank path on CPU (gloo): ranks draw different
 sequences, the reported time is the slowest rank's, and the value is the whole job's."""
+import json
 import os
 import socket
+import subprocess
 import sys
 from pathlib import Path
 
@@ -88,3 +90,46 @@ def test_sequence_sharded_gather_two_ranks_gloo(tmp_path):
     world = 2
     mp.spawn(_seq_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
     assert all((tmp_path / f"s{r}.npy").exists() for r in range(world))
+
+
+def _run_bench(*flags):
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    return subprocess.run([sys.executable, str(ROOT / "bench.py"), *flags], capture_output=True, text=True, timeout=600,
+                          env=env)
+
+
+def test_bench_launcher_starts_the_ranks_itself():
+    """`bench.py --gpus 2` outside torchrun has to start two ranks, bring them through the rendezvous and
+    the max-over-ranks reduction, and have rank 0 print ONE line with n_gpus = 2.  Rehearsed on CPU ranks
+    (gloo, no kernel, value null): the launcher, the per-rank seeding and the aggregation are the same
+    code a GPU run takes."""
+    for flags in ((), ("--shard-keys",)):
+        res = _run_bench("--gpus", "2", "--steps", "3", "--launcher-selftest", *flags)
+        assert res.returncode == 0, res.stderr[-2000:]
+        lines = [ln for ln in res.stdout.splitlines() if ln.startswith("{")]
+        assert len(lines) == 1, res.stdout
+        line = json.loads(lines[0])
+        assert line["n_gpus"] == 2 and line["gpu_launches"] == 0 and line["value"] is None
+        assert line["distinct_rank_inputs"] is True
+        assert line["stand_in_ms_max_over_ranks"] == 2.0          # ranks "took" 1 and 2 ms
+        assert line["scaling"] == ("strong" if flags else "weak")
+        if flags:
+            assert line["gathered_layout_ok"] is True
+
+
+def test_bench_refuses_to_run_fewer_ranks_than_asked():
+    """More ranks than visible GPUs: a non-zero exit and no JSON line, never a silent one-rank run."""
+    import torch
+    n = torch.cuda.device_count() + 1 if torch.cuda.is_available() else 2
+    res = _run_bench("--gpus", str(max(n, 2)), "--steps", "3")
+    assert res.returncode != 0
+    assert not [ln for ln in res.stdout.splitlines() if ln.startswith("{")]
+    assert "refusing" in res.stderr
+
+
+def test_rank_count_mismatch_under_torchrun_is_an_error():
+    env_flags = dict(RANK="0", WORLD_SIZE="1", LOCAL_RANK="0")
+    env = {**os.environ, **env_flags}
+    res = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--gpus", "2", "--launcher-selftest"], capture_output=True,
+                         text=True, timeout=300, env=env)
+    assert res.returncode != 0 and "--gpus 2" in res.stderr

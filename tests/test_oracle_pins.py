@@ -83,12 +83,13 @@ def test_three_forms_agree(oracle, seed, L, D):
 
 
 @pytest.mark.parametrize("Bc", [1, 3, 16, 64, 1000])
-def test_algorithm1_any_tile_size(oracle, Bc):
-    """Algorithm 1 with any column-tile size reproduces the two-pass result."""
+def test_single_pass_walk_any_tile_size(oracle, Bc):
+    """The single-pass tile walk of Sec. 3.3 (Algorithm 1) with any column-tile size reproduces the
+    two-pass result."""
     q, r, K, V = rand_case(9, 150, 16)
     scale = 0.5
     want = run_c(oracle, q, r, K, V, scale)
-    got = oracle.streaming_alg1(q, r, K, V, scale, Bc)
+    got = oracle.streaming_fold(q, r, K, V, scale, Bc)
     np.testing.assert_allclose(got, want, rtol=0, atol=TOL)
 
 
