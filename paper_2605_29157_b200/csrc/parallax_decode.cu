@@ -66,6 +66,9 @@ namespace {
 #ifndef PLX_L2_PROMOTION
 #define PLX_L2_PROMOTION CU_TENSOR_MAP_L2_PROMOTION_L2_256B
 #endif
+#ifndef PLX_PDL_CHAIN
+#define PLX_PDL_CHAIN 1  // launch every decode kernel as a programmatic dependent of its predecessor in the stream
+#endif
 
 constexpr int kTileKeys = 16;          // keys per warp tile (the MMA M extent)
 constexpr int kWarps = PLX_WARPS;      // warps per CTA
@@ -112,6 +115,9 @@ struct KernelParams {
     // host only: launch as a programmatic dependent of the previous kernel in the stream (the kernel's
     // first instruction waits for that kernel's results; see parallax_decode_step)
     int dependent_launch = 0;
+    // let the next kernel of the stream start early from this kernel's first instruction on (grids that fill
+    // every CTA slot of the device) instead of from its last
+    int signal_early = 0;
     // What the host knows about the buffers, for the index checks of the debug build (PLX_DEBUG_CHECKS):
     // rows each K/V tensor map covers, and the number of records `partials` has room for.
     long long kv_rows = 0;
@@ -120,6 +126,29 @@ struct KernelParams {
 
 #ifndef PLX_DEBUG_CHECKS
 #define PLX_DEBUG_CHECKS 0
+#endif
+
+// Timeline instrumentation for experiments (-DPLX_TRACE=1; never part of the shipped build): per CTA
+// the %globaltimer at start, first data, end of the tile loop and exit, plus the SM id.
+#ifndef PLX_TRACE
+#define PLX_TRACE 0
+#endif
+#if PLX_TRACE
+__device__ unsigned long long g_plx_trace[8192 * 5];
+__device__ __forceinline__ unsigned long long plx_now()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+#define PLX_STAMP(slot)                                                                  \
+    do {                                                                                 \
+        if (threadIdx.x == 0 && blockIdx.x < 8192) g_plx_trace[blockIdx.x * 5 + (slot)] = plx_now(); \
+    } while (0)
+#else
+#define PLX_STAMP(slot) \
+    do {                \
+    } while (0)
 #endif
 
 // ---------------------------------------------------------------------------
@@ -377,13 +406,47 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     const uint32_t base_addr = (raw_addr + 1023u) & ~1023u;
     uint8_t* const smem = smem_raw + (base_addr - raw_addr);
 
-    // Launched as a programmatic dependent (parallax_decode_step) this CTA may have been scheduled while
-    // the upstream-step kernel still runs: nothing that kernel produces (q, r, the appended cache row) is
-    // read before it has completed.  A no-op in an ordinary launch.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    const uint32_t ring = base_addr + warp * NSTAGES * SL::kStageBytes;
+    const uint32_t bars = base_addr + SL::kRingBytes + warp * NSTAGES * 8;
+
+    // The part of the prologue that touches no global memory: barriers and the descriptor prefetch
+    // (the tensor maps are kernel parameters).
+    if (lane == 0) {
+        if (warp == 0) {
+            prefetch_tensormap(&tmK);
+            prefetch_tensormap(&tmV);
+        }
+#pragma unroll
+        for (int s = 0; s < NSTAGES; ++s) mbar_init(bars + 8 * s, 1);
+        if (warp == 0) mbar_init(base_addr + SL::kRingBytes + kWarps * NSTAGES * 8, 1);
+        fence_barrier_init();
+    }
+    __syncwarp();
+
+    // The kernel is launched as a programmatic dependent of whatever precedes it in the stream.  If that
+    // is a kernel that lets its dependents start early (the upstream step of parallax_decode_step, the
+    // staging kernel of the host entry, the previous decode call) this CTA may be resident while it
+    // still runs: nothing it produces (q, r, an appended cache row, the workspace) is touched before
+    // it has completed and its writes are visible.  After any other kernel the wait returns at once.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // In turn, let the next kernel of the stream be scheduled before this grid has drained (it waits the
+    // same way before it touches memory), so that back-to-back decode calls overlap the next call's launch
+    // and prologue with this call's tail.  A grid that fills every CTA slot of the device signals at once:
+    // the next grid's CTAs then move in as slots free up.  A smaller grid signals at its very end instead
+    // (see the last line of the kernel): CTAs that arrive while it still runs would take the free slots
+    // beside it and could leave the next call two to an SM on part of the device with the rest idle.
+    if (p.signal_early) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    PLX_STAMP(0);
+#if PLX_TRACE
+    if (threadIdx.x == 0 && blockIdx.x < 8192) {
+        unsigned smid;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+        g_plx_trace[blockIdx.x * 5 + 4] = smid;
+    }
+#endif
+
     // stream-major order: the splits of one (sequence, KV head) are neighbours in the grid, so its
     // merge happens while other streams are still being read
     const int stream_id = blockIdx.x / p.num_splits;
@@ -436,23 +499,9 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     }
 #endif
     const int n_my = (ntiles - warp + kWarps - 1) / kWarps;  // tiles warp, warp+4, ... (may be 0)
+    // first key of this warp's tile n
+    auto tile_key = [&](int n) { return k0 + (warp + n * kWarps) * kTileKeys; };
 
-    const uint32_t ring = base_addr + warp * NSTAGES * SL::kStageBytes;
-    const uint32_t bars = base_addr + SL::kRingBytes + warp * NSTAGES * 8;
-
-    if (lane == 0) {
-        if (warp == 0) {
-            prefetch_tensormap(&tmK);
-            prefetch_tensormap(&tmV);
-        }
-#pragma unroll
-        for (int s = 0; s < NSTAGES; ++s) mbar_init(bars + 8 * s, 1);
-        if (warp == 0) mbar_init(base_addr + SL::kRingBytes + kWarps * NSTAGES * 8, 1);
-        fence_barrier_init();
-    }
-    __syncwarp();
-
-    // First cache row of this warp's tile 0; tile n of this warp starts kWarps*16*n rows later.
     const int hkv_real = hkv / p.kv_div, Hkv_real = p.Hkv / p.kv_div;
     float scale_log2e = p.scale_log2e, probe_scale = p.probe_scale, v_scale = p.v_scale;
     if constexpr (FP8) {
@@ -462,7 +511,7 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             v_scale = p.v_scales[hkv_real];
         }
     }
-    const int row0 = (b * Hkv_real + hkv_real) * p.T_max + k0 + warp * kTileKeys;
+    const int row0 = (b * Hkv_real + hkv_real) * p.T_max;  // first cache row of this stream
     // Paged cache: a 16-key tile never straddles a page (page_size is a multiple of 16), so only the
     // tile's first row changes: (page id * Hkv + hkv) * page_size + offset.  Lane 0 keeps the current
     // page id and fetches the next one a page ahead, so the lookup is off the TMA issue path.
@@ -486,8 +535,7 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     auto issue = [&](int n, int s) {
         const uint32_t bar = bars + 8 * s;
         const uint32_t dst = ring + s * SL::kStageBytes;
-        const int row = table ? paged_row(k0 + warp * kTileKeys + n * (kWarps * kTileKeys))
-                              : row0 + n * (kWarps * kTileKeys);
+        const int row = table ? paged_row(tile_key(n)) : row0 + tile_key(n);
         mbar_expect_tx(bar, SL::kStageBytes);
 #pragma unroll
         for (int h = 0; h < SL::kHalves; ++h) {
@@ -559,9 +607,11 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             failed = true;
             break;
         }
+        if (n == 0) PLX_STAMP(1);
         const uint32_t sK = ring + s * SL::kStageBytes;
         const uint32_t sV = sK + SL::kTensorBytes;
-        const int valid = k1 - (k0 + (warp + n * kWarps) * kTileKeys);  // >= 1 keys of this tile in range
+        const int key_n = tile_key(n);
+        const int valid = k1 - key_n;  // >= 1 keys of this tile in range
 
         if (valid < kTileKeys) {
             // Rows past the context may hold anything (NaN included): clear them in shared memory
@@ -610,7 +660,7 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         uint32_t pb0[NP], pb1[NP];
         // With several tokens per sequence the last lq - 1 keys are visible to the later tokens only: in the
         // few tiles that reach into them (warp-uniform test) each head of a pair gets its own key count.
-        const int to_end = L - (k0 + (warp + n * kWarps) * kTileKeys);  // keys from this tile's first to the context's last
+        const int to_end = L - key_n;  // keys from this tile's first to the context's last
         const bool per_head = to_end < kTileKeys + p.lq - 1;
 #pragma unroll
         for (int pp = 0; pp < NP; ++pp) {
@@ -737,6 +787,7 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         }
     }
 
+    PLX_STAMP(2);
     if (failed) {
         // A wait ran out: record it, give the copies still in flight one more bounded chance to
         // land before this CTA's shared memory is released, and fall through with what we have.
@@ -834,6 +885,7 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         }
     }
 
+    PLX_STAMP(3);
     if (p.mode == kModeFused) {
         // Publish this CTA's records, count the arrival, and let the CTA that completes the
         // (sequence, KV head) merge all of its splits in split order.
@@ -933,6 +985,8 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             }
         }
     }
+    // every store of this CTA has been issued: the next kernel of the stream may be scheduled
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
 // ---------------------------------------------------------------------------
@@ -1120,7 +1174,17 @@ int launch_main(const CUtensorMap& tmK, const CUtensorMap& tmV, const KernelPara
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
     const dim3 grid(static_cast<unsigned>(kp.B * kp.Hkv * kp.num_splits), 1, 1);
-    if (kp.dependent_launch) {
+    // Programmatic stream serialisation: after a kernel that signals its dependents (the previous decode
+    // call does, as do the upstream-step and staging kernels) this grid's CTAs may be scheduled before that
+    // kernel has drained (they wait before touching memory); after any other kernel the launch behaves like
+    // an ordinary one.
+    const bool chain = PLX_PDL_CHAIN || kp.dependent_launch != 0;
+    KernelParams kpl = kp;
+    {
+        int num_sms = 0;
+        kpl.signal_early = (device_sm_count(&num_sms) == PLX_OK && grid.x >= static_cast<unsigned>(num_sms) * CTAS) ? 1 : 0;
+    }
+    if (chain) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = grid;
         cfg.blockDim = dim3(kThreads, 1, 1);
@@ -1131,9 +1195,9 @@ int launch_main(const CUtensorMap& tmK, const CUtensorMap& tmV, const KernelPara
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        return cudaLaunchKernelEx(&cfg, kernel, tmK, tmV, kp) == cudaSuccess ? PLX_OK : PLX_ERR_CUDA;
+        return cudaLaunchKernelEx(&cfg, kernel, tmK, tmV, kpl) == cudaSuccess ? PLX_OK : PLX_ERR_CUDA;
     }
-    kernel<<<grid, kThreads, SL::kTotalBytes, stream>>>(tmK, tmV, kp);
+    kernel<<<grid, kThreads, SL::kTotalBytes, stream>>>(tmK, tmV, kpl);
     return cudaGetLastError() == cudaSuccess ? PLX_OK : PLX_ERR_CUDA;
 }
 
@@ -1789,6 +1853,13 @@ int parallax_decode_fwd_host(const void* q_host, const void* r_host, const void*
     if (cudaStreamSynchronize(st) != cudaSuccess) return PLX_ERR_CUDA;
     return PLX_OK;
 }
+
+#if PLX_TRACE
+int plx_trace_read(unsigned long long* host, size_t n)
+{
+    return cudaMemcpyFromSymbol(host, g_plx_trace, n * sizeof(unsigned long long)) == cudaSuccess ? PLX_OK : PLX_ERR_CUDA;
+}
+#endif
 
 int parallax_workspace_status(const void* workspace, int32_t* status_host, void* stream)
 {
