@@ -395,6 +395,12 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     // variant, so they are kept below 2^4 (P2 = P1 * S2 must stay inside the fp16 range)
     constexpr float kThreshold = FP8 ? 4.0f : kRescaleThreshold;
     constexpr int NP = (G + 1) / 2;   // GQA head pairs per KV head
+    // Up to two heads: the eight columns of a value MMA hold the pair's weights and their rounding residuals
+    // side by side, and the two halves are folded at the end.  More heads: a "quad" of four heads fills the
+    // eight columns ([P1a P1b P2a P2b | P1c P1d P2c P2d]) and the residuals go through a second MMA into the
+    // SAME accumulator, so four heads cost 32 accumulator registers per lane and eight heads 64.
+    constexpr bool SA = G > 2;
+    constexpr int NQ = SA ? (NP + 1) / 2 : 1;  // accumulator sets
     constexpr int KSTEPS = D / 16;    // k-steps of the score product
     constexpr int MTILES = D / 16;    // m-tiles of the value product
     constexpr int REC = 2 * D + 4;    // floats per partial record
@@ -549,12 +555,14 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             if (s < n_my) issue(s, s);
     }
 
-    // B fragments of [q_a q_b r_a r_b | q_c q_d r_c r_d]^T: column n = lane/4; the second head pair (G = 3, 4)
-    // takes the four columns a single pair leaves empty, so one MMA per k-step scores all four heads.
-    uint32_t bqr[KSTEPS][2];
-    {
+    // B fragments of [q_a q_b r_a r_b | q_c q_d r_c r_d]^T, one set per four heads: column n = lane/4; the
+    // second head pair of a quad takes the four columns a single pair leaves empty, so one MMA per k-step
+    // scores four heads.
+    uint32_t bqr[NQ][KSTEPS][2];
+#pragma unroll
+    for (int qd = 0; qd < NQ; ++qd) {
         const int n = lane >> 2;
-        const int hl = 2 * (n >> 2) + (n & 1);
+        const int hl = 4 * qd + 2 * (n >> 2) + (n & 1);
         const __nv_bfloat16* src = nullptr;
         if (hl < G) src = ((n & 2) ? p.r : p.q) + (static_cast<size_t>(b) * p.Hq + hkv * G + hl) * D;
 #pragma unroll
@@ -562,40 +570,45 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             if constexpr (FP8) {
                 // k-step ks, lane t: dimensions 16 ks + 4 t .. + 3 (the four bytes one ldmatrix register holds)
                 const int d = ks * 16 + (lane & 3) * 4;
-                bqr[ks][0] = src ? f16x2_from_bf16x2(*reinterpret_cast<const uint32_t*>(src + d)) : 0u;
-                bqr[ks][1] = src ? f16x2_from_bf16x2(*reinterpret_cast<const uint32_t*>(src + d + 2)) : 0u;
+                bqr[qd][ks][0] = src ? f16x2_from_bf16x2(*reinterpret_cast<const uint32_t*>(src + d)) : 0u;
+                bqr[qd][ks][1] = src ? f16x2_from_bf16x2(*reinterpret_cast<const uint32_t*>(src + d + 2)) : 0u;
             } else {
                 const int d = ks * 16 + (lane & 3) * 2;
-                bqr[ks][0] = src ? *reinterpret_cast<const uint32_t*>(src + d) : 0u;
-                bqr[ks][1] = src ? *reinterpret_cast<const uint32_t*>(src + d + 8) : 0u;
+                bqr[qd][ks][0] = src ? *reinterpret_cast<const uint32_t*>(src + d) : 0u;
+                bqr[qd][ks][1] = src ? *reinterpret_cast<const uint32_t*>(src + d + 8) : 0u;
             }
         }
     }
 
     // Running state (Algorithm 1): m in log2 units, d1, d2 as per-lane partial sums.
-    float o[NP][MTILES][4];
-    float m_run[NP][2], d1[NP][2], d2[NP][2];
+    float o[NQ][MTILES][4];
+    // Up to two heads every lane carries the one pair's state.  With more heads the four lanes of a lane quad
+    // share the pairs out (lane t computes pair t; with three pairs lane 3 repeats pair 0, with two pairs lanes
+    // 2, 3 repeat pairs 0, 1) and exchange the weights by shuffles when the P^T fragments are built.
+    float m_run[2], d1[2], d2[2];
 #pragma unroll
-    for (int pp = 0; pp < NP; ++pp) {
+    for (int e = 0; e < 2; ++e) {
+        m_run[e] = -INFINITY;
+        d1[e] = 0.0f;
+        d2[e] = 0.0f;
+    }
 #pragma unroll
-        for (int e = 0; e < 2; ++e) {
-            m_run[pp][e] = -INFINITY;
-            d1[pp][e] = 0.0f;
-            d2[pp][e] = 0.0f;
-        }
+    for (int qd = 0; qd < NQ; ++qd)
 #pragma unroll
         for (int mt = 0; mt < MTILES; ++mt)
 #pragma unroll
-            for (int j = 0; j < 4; ++j) o[pp][mt][j] = 0.0f;
-    }
+            for (int j = 0; j < 4; ++j) o[qd][mt][j] = 0.0f;
 
     // Per-lane ldmatrix geometry (byte offsets inside a swizzled [16 x 64] box).
     const int k_row = (lane & 7) + ((lane >> 3) & 1) * 8;  // K: matrices 0/1 = keys 0-7 / 8-15
     const int k_csel = lane >> 4;                          //    matrices 2/3 = next 8 columns
     const int v_row = (lane & 7) + ((lane >> 4) & 1) * 8;  // V (transposed): matrices 0/1 = keys 0-7
     const int v_csel = (lane >> 3) & 1;
-    const int role = lane & 3;       // column pair this lane feeds into P^T: 0 P1, 1 P2, 2/3 residuals
+    // column pair this lane feeds into P^T.  Up to two heads: 0 P1, 1 P2, 2/3 their residuals.  More heads:
+    // 0 P1 and 1 P2 of a quad's first pair, 2 P1 and 3 P2 of its second pair.
+    const int role = lane & 3;
     const int quad = lane & ~3;
+    const int my_pair = !SA ? 0 : NP == 4 ? role : NP == 3 ? (role == 3 ? 0 : role) : (role & 1);
     const int key_lo = lane >> 2;    // key (row of S^T) held in c[0], c[1]; c[2], c[3] hold key_lo + 8
 
     bool failed = false;
@@ -628,9 +641,11 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 
         // ---- S^T = K_c . [q r]^T ------------------------------------------------------------
         // two independent accumulator chains (even / odd k-steps) halve the dependent MMA latency
-        float c[4], c2[4];
+        float c[NQ][4], c2[NQ][4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) c[j] = c2[j] = 0.0f;
+        for (int qd = 0; qd < NQ; ++qd)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) c[qd][j] = c2[qd][j] = 0.0f;
         if constexpr (FP8) {
 #pragma unroll
             for (int kq = 0; kq < D / 32; ++kq) {  // one ldmatrix covers 16 keys x 32 dimensions = two k-steps
@@ -641,8 +656,11 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                                         e4m3x2_to_f16x2(a[0], true), e4m3x2_to_f16x2(a[1], true)};
                 const uint32_t f1[4] = {e4m3x2_to_f16x2(a[2], false), e4m3x2_to_f16x2(a[3], false),
                                         e4m3x2_to_f16x2(a[2], true), e4m3x2_to_f16x2(a[3], true)};
-                mma_f16(c, f0, bqr[2 * kq][0], bqr[2 * kq][1]);
-                mma_f16(c2, f1, bqr[2 * kq + 1][0], bqr[2 * kq + 1][1]);
+#pragma unroll
+                for (int qd = 0; qd < NQ; ++qd) {
+                    mma_f16(c[qd], f0, bqr[qd][2 * kq][0], bqr[qd][2 * kq][1]);
+                    mma_f16(c2[qd], f1, bqr[qd][2 * kq + 1][0], bqr[qd][2 * kq + 1][1]);
+                }
             }
         } else {
 #pragma unroll
@@ -650,37 +668,50 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 const int chunk = ks * 2 + k_csel;
                 uint32_t a[4];
                 ldmatrix_x4(a, sK + (chunk >> 3) * SL::kHalfBytes + k_row * 128 + (((chunk & 7) ^ (k_row & 7)) << 4));
-                mma_bf16((ks & 1) ? c2 : c, a, bqr[ks][0], bqr[ks][1]);
+#pragma unroll
+                for (int qd = 0; qd < NQ; ++qd) mma_bf16((ks & 1) ? c2[qd] : c[qd], a, bqr[qd][ks][0], bqr[qd][ks][1]);
             }
         }
 #pragma unroll
-        for (int j = 0; j < 4; ++j) c[j] += c2[j];
+        for (int qd = 0; qd < NQ; ++qd)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) c[qd][j] += c2[qd][j];
 
         // ---- online softmax state and P^T fragments -----------------------------------------
-        uint32_t pb0[NP], pb1[NP];
+        uint32_t pb0[NQ], pb1[NQ];   // P^T fragments (bf16 / fp16 parts; with up to two heads also the residuals)
+        uint32_t pr0[NQ], pr1[NQ];   // more than two heads: the rounding residuals, a second MMA into the same accumulator
         // With several tokens per sequence the last lq - 1 keys are visible to the later tokens only: in the
         // few tiles that reach into them (warp-uniform test) each head of a pair gets its own key count.
         const int to_end = L - key_n;  // keys from this tile's first to the context's last
         const bool per_head = to_end < kTileKeys + p.lq - 1;
-#pragma unroll
-        for (int pp = 0; pp < NP; ++pp) {
+        {
             int valid_a = valid, valid_b = valid;
             if (per_head) {
-                const int v0 = hkv * G + 2 * pp;
+                const int v0 = hkv * G + 2 * my_pair;
                 valid_a = min(valid, to_end - (p.lq - 1 - v0 % p.lq));
                 valid_b = min(valid, to_end - (p.lq - 1 - (v0 + 1) % p.lq));
             }
             const bool oka_lo = key_lo < valid_a, oka_hi = key_lo + 8 < valid_a;
             const bool okb_lo = key_lo < valid_b, okb_hi = key_lo + 8 < valid_b;
-            // lane 2 pp of a quad holds this pair's softmax scores (heads a, b), lane 2 pp + 1 its probe scores
-            float s1a_lo = __shfl_sync(0xffffffffu, c[0], quad + 2 * pp);
-            float s1b_lo = __shfl_sync(0xffffffffu, c[1], quad + 2 * pp);
-            float s1a_hi = __shfl_sync(0xffffffffu, c[2], quad + 2 * pp);
-            float s1b_hi = __shfl_sync(0xffffffffu, c[3], quad + 2 * pp);
-            float s2a_lo = __shfl_sync(0xffffffffu, c[0], quad + 2 * pp + 1);
-            float s2b_lo = __shfl_sync(0xffffffffu, c[1], quad + 2 * pp + 1);
-            float s2a_hi = __shfl_sync(0xffffffffu, c[2], quad + 2 * pp + 1);
-            float s2b_hi = __shfl_sync(0xffffffffu, c[3], quad + 2 * pp + 1);
+            // Of the score MMA of the pair's quad, lane 2 (pair & 1) of a lane quad holds the pair's softmax scores
+            // (heads a, b; keys key_lo and key_lo + 8) and the next lane its probe scores.
+            const int src = quad + 2 * (my_pair & 1);
+            float sc[8];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                sc[j] = __shfl_sync(0xffffffffu, c[0][j], src);
+                sc[4 + j] = __shfl_sync(0xffffffffu, c[0][j], src + 1);
+                if constexpr (NQ == 2) {
+                    const float u = __shfl_sync(0xffffffffu, c[NQ - 1][j], src);
+                    const float w = __shfl_sync(0xffffffffu, c[NQ - 1][j], src + 1);
+                    if (my_pair >> 1) {
+                        sc[j] = u;
+                        sc[4 + j] = w;
+                    }
+                }
+            }
+            float s1a_lo = sc[0], s1b_lo = sc[1], s1a_hi = sc[2], s1b_hi = sc[3];
+            float s2a_lo = sc[4], s2b_lo = sc[5], s2a_hi = sc[6], s2b_hi = sc[7];
             s1a_lo = oka_lo ? s1a_lo * scale_log2e : -INFINITY;
             s1b_lo = okb_lo ? s1b_lo * scale_log2e : -INFINITY;
             s1a_hi = oka_hi ? s1a_hi * scale_log2e : -INFINITY;
@@ -702,46 +733,81 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 ta = fmaxf(ta, __shfl_xor_sync(0xffffffffu, ta, off));
                 tb = fmaxf(tb, __shfl_xor_sync(0xffffffffu, tb, off));
             }
-            // lazy reference update (warp-uniform: every lane holds the same ta, tb, m_run)
-            if (ta > m_run[pp][0] + kThreshold || tb > m_run[pp][1] + kThreshold) {
-                const float ma = fmaxf(m_run[pp][0], ta), mb = fmaxf(m_run[pp][1], tb);
+            // Lazy reference update.  Up to two heads every lane holds the same ta, tb, m_run; with more heads
+            // they are per pair, so the warp takes the branch together as soon as any pair needs it (a pair
+            // that did not need it moves its reference to its running maximum too, which changes nothing).
+            const bool need = ta > m_run[0] + kThreshold || tb > m_run[1] + kThreshold;
+            if (SA ? __any_sync(0xffffffffu, need) : need) {
+                const float ma = fmaxf(m_run[0], ta), mb = fmaxf(m_run[1], tb);
                 // a head that has seen no key yet (and sees none in this tile) keeps its empty state
-                const float alpha_a = (ma > -INFINITY) ? fast_exp2(m_run[pp][0] - ma) : 1.0f;
-                const float alpha_b = (mb > -INFINITY) ? fast_exp2(m_run[pp][1] - mb) : 1.0f;
-                m_run[pp][0] = ma;
-                m_run[pp][1] = mb;
-                d1[pp][0] *= alpha_a;
-                d2[pp][0] *= alpha_a;
-                d1[pp][1] *= alpha_b;
-                d2[pp][1] *= alpha_b;
+                const float alpha_a = (ma > -INFINITY) ? fast_exp2(m_run[0] - ma) : 1.0f;
+                const float alpha_b = (mb > -INFINITY) ? fast_exp2(m_run[1] - mb) : 1.0f;
+                m_run[0] = ma;
+                m_run[1] = mb;
+                d1[0] *= alpha_a;
+                d2[0] *= alpha_a;
+                d1[1] *= alpha_b;
+                d2[1] *= alpha_b;
 #pragma unroll
-                for (int mt = 0; mt < MTILES; ++mt) {
-                    o[pp][mt][0] *= alpha_a;
-                    o[pp][mt][1] *= alpha_b;
-                    o[pp][mt][2] *= alpha_a;
-                    o[pp][mt][3] *= alpha_b;
+                for (int qd = 0; qd < NQ; ++qd) {
+                    float fa = alpha_a, fb = alpha_b;
+                    if constexpr (SA) {
+                        // this lane's accumulator columns of quad qd belong to pair 2 qd + (role >> 1), which lane
+                        // (quad + that pair) computes; a pair that does not exist has all-zero columns
+                        const int owner = quad + min(2 * qd + (role >> 1), NP - 1);
+                        fa = __shfl_sync(0xffffffffu, alpha_a, owner);
+                        fb = __shfl_sync(0xffffffffu, alpha_b, owner);
+                    }
+#pragma unroll
+                    for (int mt = 0; mt < MTILES; ++mt) {
+                        o[qd][mt][0] *= fa;
+                        o[qd][mt][1] *= fb;
+                        o[qd][mt][2] *= fa;
+                        o[qd][mt][3] *= fb;
+                    }
                 }
             }
             // reference 0 while a head has seen nothing: its scores are all -inf and its weights exact zeros
-            const float ref_a = (m_run[pp][0] > -INFINITY) ? m_run[pp][0] : 0.0f;
-            const float ref_b = (m_run[pp][1] > -INFINITY) ? m_run[pp][1] : 0.0f;
+            const float ref_a = (m_run[0] > -INFINITY) ? m_run[0] : 0.0f;
+            const float ref_b = (m_run[1] > -INFINITY) ? m_run[1] : 0.0f;
             const float p1a_lo = fast_exp2(s1a_lo - ref_a);
             const float p1b_lo = fast_exp2(s1b_lo - ref_b);
             const float p1a_hi = fast_exp2(s1a_hi - ref_a);
             const float p1b_hi = fast_exp2(s1b_hi - ref_b);
             const float p2a_lo = p1a_lo * s2a_lo, p2b_lo = p1b_lo * s2b_lo;
             const float p2a_hi = p1a_hi * s2a_hi, p2b_hi = p1b_hi * s2b_hi;
-            d1[pp][0] += p1a_lo + p1a_hi;
-            d1[pp][1] += p1b_lo + p1b_hi;
-            d2[pp][0] += p2a_lo + p2a_hi;
-            d2[pp][1] += p2b_lo + p2b_hi;
-            const bool second = role & 1, resid = role & 2;
-            const uint32_t f_lo = FP8 ? pack_f16_pair(second ? p2a_lo : p1a_lo, second ? p2b_lo : p1b_lo, resid)
-                                      : pack_bf16_pair(second ? p2a_lo : p1a_lo, second ? p2b_lo : p1b_lo, resid);
-            const uint32_t f_hi = FP8 ? pack_f16_pair(second ? p2a_hi : p1a_hi, second ? p2b_hi : p1b_hi, resid)
-                                      : pack_bf16_pair(second ? p2a_hi : p1a_hi, second ? p2b_hi : p1b_hi, resid);
-            pb0[pp] = movmatrix_trans(f_lo);   // keys 0-7  -> k rows 0-7 of the B operand
-            pb1[pp] = movmatrix_trans(f_hi);   // keys 8-15 -> k rows 8-15
+            d1[0] += p1a_lo + p1a_hi;
+            d1[1] += p1b_lo + p1b_hi;
+            d2[0] += p2a_lo + p2a_hi;
+            d2[1] += p2b_lo + p2b_hi;
+            const bool second = role & 1;
+            if constexpr (!SA) {
+                const bool resid = role & 2;
+                const uint32_t f_lo = FP8 ? pack_f16_pair(second ? p2a_lo : p1a_lo, second ? p2b_lo : p1b_lo, resid)
+                                          : pack_bf16_pair(second ? p2a_lo : p1a_lo, second ? p2b_lo : p1b_lo, resid);
+                const uint32_t f_hi = FP8 ? pack_f16_pair(second ? p2a_hi : p1a_hi, second ? p2b_hi : p1b_hi, resid)
+                                          : pack_bf16_pair(second ? p2a_hi : p1a_hi, second ? p2b_hi : p1b_hi, resid);
+                pb0[0] = movmatrix_trans(f_lo);   // keys 0-7  -> k rows 0-7 of the B operand
+                pb1[0] = movmatrix_trans(f_hi);   // keys 8-15 -> k rows 8-15
+            } else {
+#pragma unroll
+                for (int qd = 0; qd < NQ; ++qd) {
+                    // column pair (role) of quad qd: P1 (even role) or P2 (odd role) of pair 2 qd + (role >> 1)
+                    const int want = 2 * qd + (role >> 1);
+                    const int owner = quad + min(want, NP - 1);
+                    const float g1a_lo = __shfl_sync(0xffffffffu, p1a_lo, owner), g2a_lo = __shfl_sync(0xffffffffu, p2a_lo, owner);
+                    const float g1b_lo = __shfl_sync(0xffffffffu, p1b_lo, owner), g2b_lo = __shfl_sync(0xffffffffu, p2b_lo, owner);
+                    const float g1a_hi = __shfl_sync(0xffffffffu, p1a_hi, owner), g2a_hi = __shfl_sync(0xffffffffu, p2a_hi, owner);
+                    const float g1b_hi = __shfl_sync(0xffffffffu, p1b_hi, owner), g2b_hi = __shfl_sync(0xffffffffu, p2b_hi, owner);
+                    const bool exists = want < NP;
+                    const float ya_lo = exists ? (second ? g2a_lo : g1a_lo) : 0.0f, yb_lo = exists ? (second ? g2b_lo : g1b_lo) : 0.0f;
+                    const float ya_hi = exists ? (second ? g2a_hi : g1a_hi) : 0.0f, yb_hi = exists ? (second ? g2b_hi : g1b_hi) : 0.0f;
+                    pb0[qd] = movmatrix_trans(FP8 ? pack_f16_pair(ya_lo, yb_lo, false) : pack_bf16_pair(ya_lo, yb_lo, false));
+                    pb1[qd] = movmatrix_trans(FP8 ? pack_f16_pair(ya_hi, yb_hi, false) : pack_bf16_pair(ya_hi, yb_hi, false));
+                    pr0[qd] = movmatrix_trans(FP8 ? pack_f16_pair(ya_lo, yb_lo, true) : pack_bf16_pair(ya_lo, yb_lo, true));
+                    pr1[qd] = movmatrix_trans(FP8 ? pack_f16_pair(ya_hi, yb_hi, true) : pack_bf16_pair(ya_hi, yb_hi, true));
+                }
+            }
         }
 
         // ---- O^T += V_c^T . P^T -------------------------------------------------------------
@@ -761,19 +827,37 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 const uint32_t f1[4] = {e4m3x2_to_f16x2(x[1], false), e4m3x2_to_f16x2(x[1], true),
                                         e4m3x2_to_f16x2(x[3], false), e4m3x2_to_f16x2(x[3], true)};
 #pragma unroll
-                for (int pp = 0; pp < NP; ++pp) {
-                    mma_f16(o[pp][2 * mq], f0, pb0[pp], pb1[pp]);
-                    mma_f16(o[pp][2 * mq + 1], f1, pb0[pp], pb1[pp]);
+                for (int qd = 0; qd < NQ; ++qd) {
+                    mma_f16(o[qd][2 * mq], f0, pb0[qd], pb1[qd]);
+                    mma_f16(o[qd][2 * mq + 1], f1, pb0[qd], pb1[qd]);
+                }
+                if constexpr (SA) {
+#pragma unroll
+                    for (int qd = 0; qd < NQ; ++qd) {
+                        mma_f16(o[qd][2 * mq], f0, pr0[qd], pr1[qd]);
+                        mma_f16(o[qd][2 * mq + 1], f1, pr0[qd], pr1[qd]);
+                    }
                 }
             }
         } else {
 #pragma unroll
-            for (int mt = 0; mt < MTILES; ++mt) {
-                const int chunk = mt * 2 + v_csel;
-                uint32_t a[4];
-                ldmatrix_x4_trans(a, sV + (chunk >> 3) * SL::kHalfBytes + v_row * 128 + (((chunk & 7) ^ (v_row & 7)) << 4));
+            for (int mt = 0; mt < MTILES; mt += 2) {  // two m-tiles at a time: the residual MMAs follow two others
+                uint32_t a0[4], a1[4];
+                const int ch0 = mt * 2 + v_csel, ch1 = ch0 + 2;
+                ldmatrix_x4_trans(a0, sV + (ch0 >> 3) * SL::kHalfBytes + v_row * 128 + (((ch0 & 7) ^ (v_row & 7)) << 4));
+                ldmatrix_x4_trans(a1, sV + (ch1 >> 3) * SL::kHalfBytes + v_row * 128 + (((ch1 & 7) ^ (v_row & 7)) << 4));
 #pragma unroll
-                for (int pp = 0; pp < NP; ++pp) mma_bf16(o[pp][mt], a, pb0[pp], pb1[pp]);
+                for (int qd = 0; qd < NQ; ++qd) {
+                    mma_bf16(o[qd][mt], a0, pb0[qd], pb1[qd]);
+                    mma_bf16(o[qd][mt + 1], a1, pb0[qd], pb1[qd]);
+                }
+                if constexpr (SA) {
+#pragma unroll
+                    for (int qd = 0; qd < NQ; ++qd) {
+                        mma_bf16(o[qd][mt], a0, pr0[qd], pr1[qd]);
+                        mma_bf16(o[qd][mt + 1], a1, pr0[qd], pr1[qd]);
+                    }
+                }
             }
         }
 
@@ -803,45 +887,49 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 
     // ---- per-warp wrap-up: finish the lane-partial sums, fold residual columns ----------------
 #pragma unroll
-    for (int pp = 0; pp < NP; ++pp) {
+    for (int e = 0; e < 2; ++e) {
 #pragma unroll
-        for (int e = 0; e < 2; ++e) {
-#pragma unroll
-            for (int off = 4; off < 32; off <<= 1) {
-                d1[pp][e] += __shfl_xor_sync(0xffffffffu, d1[pp][e], off);
-                d2[pp][e] += __shfl_xor_sync(0xffffffffu, d2[pp][e], off);
-            }
+        for (int off = 4; off < 32; off <<= 1) {
+            d1[e] += __shfl_xor_sync(0xffffffffu, d1[e], off);
+            d2[e] += __shfl_xor_sync(0xffffffffu, d2[e], off);
         }
+    }
+    if constexpr (!SA) {  // up to two heads: columns 4-7 accumulated the residual products
 #pragma unroll
         for (int mt = 0; mt < MTILES; ++mt)
 #pragma unroll
-            for (int j = 0; j < 4; ++j) o[pp][mt][j] += __shfl_xor_sync(0xffffffffu, o[pp][mt][j], 2);
+            for (int j = 0; j < 4; ++j) o[0][mt][j] += __shfl_xor_sync(0xffffffffu, o[0][mt][j], 2);
     }
 
     __syncthreads();  // every warp has drained its ring: reuse it as merge scratch
     float* const scratch = reinterpret_cast<float*>(smem);
-#pragma unroll
-    for (int pp = 0; pp < NP; ++pp) {
-        float* rec_a = scratch + ((warp * NP + pp) * 2 + 0) * REC;
+    if (lane < NP) {  // lanes 0 .. NP-1 hold the state of pairs 0 .. NP-1
+        float* rec_a = scratch + ((warp * NP + lane) * 2 + 0) * REC;
         float* rec_b = rec_a + REC;
-        if (lane == 0) {
-            rec_a[0] = m_run[pp][0];
-            rec_a[1] = d1[pp][0];
-            rec_a[2] = d2[pp][0];
-            rec_b[0] = m_run[pp][1];
-            rec_b[1] = d1[pp][1];
-            rec_b[2] = d2[pp][1];
-        }
-        if (role < 2) {  // role 0 holds O1 columns, role 1 holds O2 columns
+        rec_a[0] = m_run[0];
+        rec_a[1] = d1[0];
+        rec_a[2] = d2[0];
+        rec_b[0] = m_run[1];
+        rec_b[1] = d1[1];
+        rec_b[2] = d2[1];
+    }
+#pragma unroll
+    for (int qd = 0; qd < NQ; ++qd) {
+        // Up to two heads: role 0 holds the pair's O1 columns, role 1 its O2 columns.  More heads: roles 0, 1
+        // hold O1, O2 of the quad's first pair, roles 2, 3 those of its second pair.
+        const int pp = SA ? 2 * qd + (role >> 1) : 0;
+        if (SA ? pp < NP : role < 2) {
+            float* rec_a = scratch + ((warp * NP + pp) * 2 + 0) * REC;
+            float* rec_b = rec_a + REC;
             // accumulator rows g and g + 8 of an m-tile are dimensions g, g + 8 (2g, 2g + 1 in the FP8 variant)
-            const int off = 4 + role * D + (FP8 ? 2 * key_lo : key_lo);
+            const int off = 4 + (role & 1) * D + (FP8 ? 2 * key_lo : key_lo);
             constexpr int kUp = FP8 ? 1 : 8;
 #pragma unroll
             for (int mt = 0; mt < MTILES; ++mt) {
-                rec_a[off + mt * 16] = o[pp][mt][0];
-                rec_b[off + mt * 16] = o[pp][mt][1];
-                rec_a[off + mt * 16 + kUp] = o[pp][mt][2];
-                rec_b[off + mt * 16 + kUp] = o[pp][mt][3];
+                rec_a[off + mt * 16] = o[qd][mt][0];
+                rec_b[off + mt * 16] = o[qd][mt][1];
+                rec_a[off + mt * 16 + kUp] = o[qd][mt][2];
+                rec_b[off + mt * 16 + kUp] = o[qd][mt][3];
             }
         }
     }
@@ -1060,14 +1148,14 @@ size_t partial_bytes(int B, int Hq, int D, int splits)
 
 bool shape_ok(int B, int Hq, int Hkv, int D) { return B > 0 && Hq > 0 && Hkv > 0 && D > 0 && Hq % Hkv == 0; }
 // Query heads per CTA (g <= 4) and CTAs ("virtual KV heads") per real KV head for a group of G query heads.
-void split_group(int G, int* g, int* kv_div)
+void split_group(int G, int* g, int* kv_div, int max_g = 8)
 {
-    if (G <= 4) *g = G;
-    else if (G % 4 == 0) *g = 4;
-    else if (G % 3 == 0) *g = 3;
-    else if (G % 2 == 0) *g = 2;
-    else *g = 1;
-    *kv_div = G / *g;
+    // the largest group size up to max_g that divides G (the kernel is built for 1 .. 8 heads per CTA)
+    int best = 1;
+    for (int c = 1; c <= max_g && c <= G; ++c)
+        if (G % c == 0) best = c;
+    *g = best;
+    *kv_div = G / best;
 }
 bool shape_supported(int Hq, int Hkv, int D)
 {
@@ -1075,18 +1163,18 @@ bool shape_supported(int Hq, int Hkv, int D)
     return (D == 64 || D == 128) && G >= 1 && G <= 64;
 }
 // Rewrites the launch parameters for group sizes above 4 and returns the per-CTA group size.
-int apply_group(KernelParams* kp, int Hq, int Hkv)
+int apply_group(KernelParams* kp, int Hq, int Hkv, int max_g = 8)
 {
     int g = 1, kv_div = 1;
-    split_group(Hq / Hkv, &g, &kv_div);
+    split_group(Hq / Hkv, &g, &kv_div, max_g);
     kp->Hkv = Hkv * kv_div;
     kp->kv_div = kv_div;
     return g;
 }
-int virtual_kv_heads(int Hq, int Hkv)
+int virtual_kv_heads(int Hq, int Hkv, int max_g = 8)
 {
     int g = 1, kv_div = 1;
-    split_group(Hq / Hkv, &g, &kv_div);
+    split_group(Hq / Hkv, &g, &kv_div, max_g);
     return Hkv * kv_div;
 }
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
@@ -1231,33 +1319,36 @@ int dispatch_main(int D, int G, const CUtensorMap& tmK, const CUtensorMap& tmV, 
     // CTAs per SM) two stages per warp measured fastest (128 KiB in flight per SM: deeper rings only
     // lengthen the memory queues); smaller grids keep three stages, each CTA then needs more in flight.
     const long long ctas = static_cast<long long>(kp.B) * kp.Hkv * kp.num_splits;
+    // Five to eight heads per CTA keep two accumulator sets (64 registers per lane at D = 128, 32 at D = 64):
+    // about 220 / 152 registers per thread, i.e. two CTAs per SM at D = 128 and three at D = 64.
+#define PLX_LAUNCH_G(DD, ST, CT, CT_BIG)                                                     \
+    switch (G) {                                                                             \
+        case 1: return launch_main<DD, 1, ST, CT>(tmK, tmV, kp, stream);                     \
+        case 2: return launch_main<DD, 2, ST, CT>(tmK, tmV, kp, stream);                     \
+        case 3: return launch_main<DD, 3, ST, CT>(tmK, tmV, kp, stream);                     \
+        case 4: return launch_main<DD, 4, ST, CT>(tmK, tmV, kp, stream);                     \
+        case 5: return launch_main<DD, 5, ST, CT_BIG>(tmK, tmV, kp, stream);                 \
+        case 6: return launch_main<DD, 6, ST, CT_BIG>(tmK, tmV, kp, stream);                 \
+        case 7: return launch_main<DD, 7, ST, CT_BIG>(tmK, tmV, kp, stream);                 \
+        case 8: return launch_main<DD, 8, ST, CT_BIG>(tmK, tmV, kp, stream);                 \
+        default: return PLX_ERR_UNSUPPORTED;                                                 \
+    }
     if (D == 128) {
         const bool two_stage = kp.chunk_len <= PLX_TWO_STAGE_MAX_CHUNK;
         if (two_stage) {
-            if (G == 1) return launch_main<128, 1, 2>(tmK, tmV, kp, stream);
-            if (G == 2) return launch_main<128, 2, 2>(tmK, tmV, kp, stream);
-            if (G == 3) return launch_main<128, 3, 2>(tmK, tmV, kp, stream);
-            if (G == 4) return launch_main<128, 4, 2>(tmK, tmV, kp, stream);
+            PLX_LAUNCH_G(128, 2, kCtasPerSm, kCtasPerSm)
         }
-        if (G == 1) return launch_main<128, 1, PLX_STAGES_D128>(tmK, tmV, kp, stream);
-        if (G == 2) return launch_main<128, 2, PLX_STAGES_D128>(tmK, tmV, kp, stream);
-        if (G == 3) return launch_main<128, 3, PLX_STAGES_D128>(tmK, tmV, kp, stream);
-        if (G == 4) return launch_main<128, 4, PLX_STAGES_D128>(tmK, tmV, kp, stream);
+        PLX_LAUNCH_G(128, PLX_STAGES_D128, kCtasPerSm, kCtasPerSm)
     } else if (D == 64) {
         int num_sms = 0;
         if (int rc = device_sm_count(&num_sms); rc != PLX_OK) return rc;
         const bool two_stage = kp.chunk_len <= 2 * kChunkGranule || ctas >= 3LL * num_sms;
         if (two_stage) {
-            if (G == 1) return launch_main<64, 1, 2, PLX_CTAS_PER_SM_D64>(tmK, tmV, kp, stream);
-            if (G == 2) return launch_main<64, 2, 2, PLX_CTAS_PER_SM_D64>(tmK, tmV, kp, stream);
-            if (G == 3) return launch_main<64, 3, 2, PLX_CTAS_PER_SM_D64>(tmK, tmV, kp, stream);
-            if (G == 4) return launch_main<64, 4, 2, PLX_CTAS_PER_SM_D64>(tmK, tmV, kp, stream);
+            PLX_LAUNCH_G(64, 2, PLX_CTAS_PER_SM_D64, 3)
         }
-        if (G == 1) return launch_main<64, 1, PLX_STAGES_D64, PLX_CTAS_PER_SM_D64>(tmK, tmV, kp, stream);
-        if (G == 2) return launch_main<64, 2, PLX_STAGES_D64, PLX_CTAS_PER_SM_D64>(tmK, tmV, kp, stream);
-        if (G == 3) return launch_main<64, 3, PLX_STAGES_D64, PLX_CTAS_PER_SM_D64>(tmK, tmV, kp, stream);
-        if (G == 4) return launch_main<64, 4, PLX_STAGES_D64, PLX_CTAS_PER_SM_D64>(tmK, tmV, kp, stream);
+        PLX_LAUNCH_G(64, PLX_STAGES_D64, PLX_CTAS_PER_SM_D64, 3)
     }
+#undef PLX_LAUNCH_G
     return PLX_ERR_UNSUPPORTED;
 }
 
@@ -1458,7 +1549,7 @@ static int decode_fwd_impl(const void* q, const void* r, const void* k_cache, co
     if (num_splits == 0) {
         int sms = 0;
         if ((rc = device_sm_count(&sms)) != PLX_OK) return rc;
-        plan_splits(B, virtual_kv_heads(Hq, Hkv), D, T_max, sms, seqlens != nullptr, &chunk_len, &ns, fp8);
+        plan_splits(B, virtual_kv_heads(Hq, Hkv, fp8 ? 4 : 8), D, T_max, sms, seqlens != nullptr, &chunk_len, &ns, fp8);
         // never plan beyond what the caller's workspace can hold
         if (ns > 1) {
             const size_t fixed = fixed_bytes(B, Hq, D);
@@ -1503,10 +1594,11 @@ static int decode_fwd_impl(const void* q, const void* r, const void* k_cache, co
     }
     kp.dependent_launch = dependent_launch ? 1 : 0;
     kp.lq = lq;
+    const int max_g = fp8 ? 4 : 8;  // the e4m3 variant is built for up to four heads per CTA
     kp.kv_rows = static_cast<long long>(rows);
     if (partials)
         kp.partial_records = static_cast<long long>((workspace_bytes - fixed_bytes(B, Hq, D)) / ((2 * D + 4) * sizeof(float)));
-    const int g = apply_group(&kp, Hq, Hkv);
+    const int g = apply_group(&kp, Hq, Hkv, max_g);
     return dispatch_main(D, g, tmK, tmV, kp, st, fp8);
 }
 
