@@ -385,7 +385,7 @@ def run_ours(args, rank, world, local_rank):
     t_call = timer.run(step, args.steps)
     ms_per_step = t_call["ms_per_step"]
     # one launch per call, except steps the library hands to the tensor-core kernel (more than eight rows per KV head)
-    launches_per_step = tensor_core_launches(cfg, Lq, sms) if cfg.G * Lq > 8 and not (args.fp8_kv or args.page_size) else 1
+    launches_per_step = tensor_core_launches(cfg, Lq, sms) if routed_to_tensor_core(cfg, Lq) and not (args.fp8_kv or args.page_size) else 1
     value = whole_job_value(kv_bytes, world, ms_per_step)
     assert plx.parallax_workspace_status(ws) == 0, "device-side wait timed out"
     us_graph = graph_replay_us(step, nsets)
@@ -485,6 +485,20 @@ def run_ours(args, rank, world, local_rank):
                                   "single_thread_C2": single_thread_oracle_c2()}
     sampler.close()
     return result
+
+
+def routed_to_tensor_core(cfg, Lq):
+    """Mirrors the library's routing of a multi-token step (only to count launches): up to eight rows per KV head
+    run on the decode kernel, nine to sixteen too when they split into two CTAs of at most eight rows and the call
+    has at least 128 (sequence, KV head) streams, everything else on the tensor-core kernel."""
+    rows = cfg.G * Lq
+    if rows <= 8:
+        return False
+    if rows <= 16 and cfg.B * cfg.Hkv >= 128:
+        g = max(c for c in range(1, 9) if rows % c == 0)
+        if rows // g <= 2:
+            return False
+    return True
 
 
 def tensor_core_launches(cfg, Lq, sms):

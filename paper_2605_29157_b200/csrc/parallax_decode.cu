@@ -1638,9 +1638,19 @@ int parallax_decode_fwd_fp8(const void* q, const void* r, const void* k_cache, c
                            workspace_bytes, num_splits, stream, nullptr, 0, 0, 0, true, k_scale, v_scale);
 }
 
-// Rows per KV head from which a multi-token step goes to the tensor-core kernel (measured crossover: up to
-// eight rows the decode kernel is as fast or faster at every batch size, from sixteen on it loses everywhere).
-constexpr int kMultiTokenDecodeRows = 8;
+// Which kernel takes a step of `rows` = (query heads per KV head) x (new tokens) rows per KV head.  Up to eight
+// rows one CTA of the decode kernel serves a KV head and is the faster route at every batch size.  Nine to sixteen
+// rows that split into two CTAs of at most eight (10 = 2 x 5, 12, 14, 16) stay on the decode kernel when the call has
+// at least 128 (sequence, KV head) streams: measured at 10 / 12 / 16 rows, context 8192, 8 KV heads: batch 64
+// 505 / 525 / 533 us against 728 / 754 / 795 us on the tensor-core kernel, batch 16 132 / 131 / 142 against
+// 187 / 188 / 208; batch 8 128 / 128 / 121 against 115 / 115 / 101 (the tensor-core kernel's split-KV wins there).
+// From 24 rows on the tensor-core kernel is faster or equal everywhere.
+#ifndef PLX_MULTI_TOKEN_DECODE_ROWS
+#define PLX_MULTI_TOKEN_DECODE_ROWS 8
+#endif
+constexpr int kMultiTokenDecodeRows = PLX_MULTI_TOKEN_DECODE_ROWS;
+constexpr int kTwoCtaDecodeRows = 16;
+constexpr long long kTwoCtaDecodeMinStreams = 128;
 // The part of a decode workspace that holds split records (after the status word, counters and staging).
 static void records_region(void* workspace, size_t workspace_bytes, int B, int rows, int D, void** rec, size_t* rec_bytes)
 {
@@ -1648,11 +1658,18 @@ static void records_region(void* workspace, size_t workspace_bytes, int B, int r
     *rec = (workspace && workspace_bytes > fixed) ? static_cast<uint8_t*>(workspace) + fixed : nullptr;
     *rec_bytes = *rec ? workspace_bytes - fixed : 0;
 }
-static bool use_tensor_core_kernel(const void* q, const void* r, const void* out, int Hq, int Hkv, int Lq, int D)
+static bool use_tensor_core_kernel(const void* q, const void* r, const void* out, int B, int Hq, int Hkv, int Lq, int D)
 {
     const long long rows = static_cast<long long>(Hq / Hkv) * Lq;
     const bool can = aligned(q, 16) && aligned(r, 16) && aligned(out, 16) && (D == 64 || D == 128);
-    return rows > 64 || (rows > kMultiTokenDecodeRows && can);
+    if (rows > 64) return true;
+    if (!can || rows <= kMultiTokenDecodeRows) return false;
+    if (rows <= kTwoCtaDecodeRows && static_cast<long long>(B) * Hkv >= kTwoCtaDecodeMinStreams) {
+        int g = 1, kv_div = 1;
+        split_group(static_cast<int>(rows), &g, &kv_div);
+        if (kv_div <= 2) return false;
+    }
+    return true;
 }
 
 int parallax_decode_fwd_multi(const void* q, const void* r, const void* k_cache, const void* v_cache,
@@ -1662,7 +1679,7 @@ int parallax_decode_fwd_multi(const void* q, const void* r, const void* k_cache,
 {
     if (Lq <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || B <= 0) return PLX_ERR_BAD_SHAPE;
     if (workspace && !aligned(workspace, 16)) return PLX_ERR_ALIGNMENT;
-    if (use_tensor_core_kernel(q, r, out, Hq, Hkv, Lq, D)) {
+    if (use_tensor_core_kernel(q, r, out, B, Hq, Hkv, Lq, D)) {
         void* rec = nullptr;
         size_t rec_bytes = 0;
         records_region(workspace, workspace_bytes, B, Hq * Lq, D, &rec, &rec_bytes);
@@ -1751,7 +1768,7 @@ int parallax_decode_fwd_multi_paged(const void* q, const void* r, const void* k_
     if (workspace && !aligned(workspace, 16)) return PLX_ERR_ALIGNMENT;
     if (num_pages <= 0 || page_size <= 0 || page_size % kTileKeys != 0 || max_pages_per_seq <= 0)
         return PLX_ERR_BAD_SHAPE;
-    if (page_size % 64 == 0 && use_tensor_core_kernel(q, r, out, Hq, Hkv, Lq, D)) {  // that kernel walks 64-key tiles
+    if (page_size % 64 == 0 && use_tensor_core_kernel(q, r, out, B, Hq, Hkv, Lq, D)) {  // that kernel walks 64-key tiles
         void* rec = nullptr;
         size_t rec_bytes = 0;
         records_region(workspace, workspace_bytes, B, Hq * Lq, D, &rec, &rec_bytes);
