@@ -196,6 +196,61 @@ def test_backward_full_size_in_the_bench_configuration(plx, oracle):
     assert ((dvf.sum(dim=2) - want_sum).abs() <= 2e-3 * dvf.abs().sum(dim=2)).all()
 
 
+def test_backward_full_size_long_sequence(plx, oracle):
+    """T2 (two sequences of 16384 tokens) at full size with the bench's dtypes.  dq, dr on sampled rows.  dk, dv
+    of the LAST 256 keys of one (sequence, KV head) group: only the last 256 rows see those keys, so the oracle's
+    backward of those rows alone (a 256-token problem on the full context) gives their complete gradients.
+    Every group by the two shift invariances."""
+    cfg, Lq = wl.BACKWARD_CONFIGS["T2"]
+    B, Hq, Hkv, D, T, G = cfg.B, cfg.Hq, cfg.Hkv, cfg.D, cfg.T_max, cfg.G
+    x = wl.make_prefill_inputs(cfg, Lq, "cuda")
+    gen = torch.Generator(device="cuda").manual_seed(cfg.seed + 5)
+    dout = torch.randn(B, Hq, Lq, D, device="cuda", generator=gen).to(torch.bfloat16)
+    out = torch.empty(B, Hq, Lq, D, dtype=torch.bfloat16, device="cuda")
+    vbar = torch.empty_like(out)
+    lse = torch.empty(B, Hq, Lq, dtype=torch.float32, device="cuda")
+    tbar = torch.empty_like(lse)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    plx.parallax_prefill_fwd_save(x["q"], x["r"], x["k"], x["v"], None, out, lse, tbar, vbar, cfg.scale, status)
+    dq, dr = torch.empty_like(out), torch.empty_like(out)
+    dk = torch.empty(B, Hkv, T, D, dtype=torch.bfloat16, device="cuda")
+    dv = torch.empty_like(dk)
+    ws = torch.empty(plx.parallax_prefill_bwd_workspace_bytes(B, Hq, Lq), dtype=torch.uint8, device="cuda")
+    plx.parallax_prefill_bwd(x["q"], x["r"], x["k"], x["v"], dout, out, lse, tbar, vbar, None, dq, dr, dk, dv,
+                             cfg.scale, ws, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+
+    g = np.random.default_rng(17)
+    rows = [(int(g.integers(B)), int(g.integers(Hq)), int(i)) for i in
+            list(g.integers(0, Lq, size=12)) + [0, 127, 128, Lq - 1]]
+    got_q, got_r, want_q, want_r = [], [], [], []
+    for (b, h, i) in rows:
+        hkv = h // G
+        one = lambda t: wl.bf16_bits(t[b:b + 1, h:h + 1, i:i + 1])
+        kb, vb = wl.bf16_bits(x["k"][b:b + 1, hkv:hkv + 1, :i + 1]), wl.bf16_bits(x["v"][b:b + 1, hkv:hkv + 1, :i + 1])
+        wq, wr, _, _ = oracle.backward_bf16(one(x["q"]), one(x["r"]), kb, vb, one(dout), None, cfg.scale)
+        want_q.append(wq[0, 0, 0])
+        want_r.append(wr[0, 0, 0])
+        got_q.append(dq[b, h, i].float().cpu().numpy())
+        got_r.append(dr[b, h, i].float().cpu().numpy())
+    check_grad("dq (sampled rows)", np.stack(got_q), np.stack(want_q))
+    check_grad("dr (sampled rows)", np.stack(got_r), np.stack(want_r))
+
+    b, hkv, tail = 1, 6, 256
+    hs = slice(hkv * G, (hkv + 1) * G)
+    last = lambda t: wl.bf16_bits(t[b:b + 1, hs, Lq - tail:])
+    kb, vb = wl.bf16_bits(x["k"][b:b + 1, hkv:hkv + 1]), wl.bf16_bits(x["v"][b:b + 1, hkv:hkv + 1])
+    _, _, wk, wv = oracle.backward_bf16(last(x["q"]), last(x["r"]), kb, vb, last(dout), None, cfg.scale)
+    check_grad("dk (last keys of one group)", dk[b, hkv, T - tail:].float().cpu().numpy(), wk[0, 0, T - tail:])
+    check_grad("dv (last keys of one group)", dv[b, hkv, T - tail:].float().cpu().numpy(), wv[0, 0, T - tail:])
+
+    dkf, dvf = dk.float(), dv.float()
+    assert (dkf.sum(dim=2).abs() <= 2e-3 * dkf.abs().sum(dim=2)).all()
+    want_sum = dout.float().reshape(B, Hkv, G, Lq, D).sum(dim=(2, 3))
+    assert ((dvf.sum(dim=2) - want_sum).abs() <= 2e-3 * dvf.abs().sum(dim=2)).all()
+
+
 def test_autograd_front_end(plx, oracle):
     """torch.autograd wrapper: out.backward() routes to the library's backward; gradients against the oracle."""
     from paper_2605_29157_b200.autograd import parallax_attention

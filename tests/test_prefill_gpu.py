@@ -107,20 +107,24 @@ def test_prefill_plain_bf16_weights(plx, oracle):
     assert e["max_abs"] <= MAX_ABS_TOL and e["mean_abs"] <= MEAN_ABS_TOL and e["rel_rms"] <= 1e-2, e
 
 
-@pytest.mark.parametrize("name", ["P1", "P3"])
+@pytest.mark.parametrize("name", ["P1", "P2", "P3", "P4"])
 def test_prefill_full_size_in_the_bench_configuration(plx, oracle, name):
-    """Full-size prefill workloads with the launch configuration and dtypes the bench times (bf16
-    output), checked on sampled rows: each row is a one-token problem for the oracle."""
+    """Full-size prefill workloads with the entry point, workspace and dtypes the bench times (bf16 output;
+    P4's few row tiles make the library divide the keys among CTAs and finish with its merge kernel),
+    checked on sampled rows: each row is a one-token problem for the oracle."""
     cfg, Lq = wl.PREFILL_CONFIGS[name]
     x = wl.make_prefill_inputs(cfg, Lq, "cuda")
-    out = torch.empty(cfg.B, cfg.Hq, Lq, cfg.D, dtype=torch.bfloat16, device="cuda")
+    out = torch.full((cfg.B, cfg.Hq, Lq, cfg.D), float("nan"), dtype=torch.bfloat16, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    plx.parallax_prefill_fwd(x["q"], x["r"], x["k"], x["v"], None, out, cfg.scale, status)
+    ws = torch.empty(min(plx.parallax_prefill_workspace_bytes(cfg.B, cfg.Hq, cfg.D, Lq, 64), 1 << 30), dtype=torch.uint8,
+                     device="cuda")
+    plx.parallax_prefill_fwd_ex(x["q"], x["r"], x["k"], x["v"], None, out, cfg.scale, ws, 0, status)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
+    assert torch.isfinite(out.float()).all()
     g = np.random.default_rng(11)
     rows = [(int(g.integers(cfg.B)), int(g.integers(cfg.Hq)), int(i)) for i in
-            list(g.integers(0, Lq, size=40)) + [0, 1, 63, 64, 127, 128, Lq - 1]]
+            list(g.integers(0, Lq, size=40)) + [i for i in (0, 1, 63, 64, 127, 128, Lq - 1) if i < Lq]]
     for (b, h, i) in rows:
         n = cfg.T_max - Lq + i + 1
         hkv = h // cfg.G
