@@ -262,7 +262,9 @@ int parallax_prefill_fwd(const void* q, const void* r, const void* k_cache, cons
  * result is the Parallax output for the dequantised cache (k_scale * k8, v_scale * v8): e4m3 converts
  * exactly to fp16, the products run as fp16 x fp16 -> fp32 MMAs (q and r are converted bf16 -> fp16:
  * exact for magnitudes in [6.1e-5, 65504]), the weights reach the value product as fp16 plus fp16
- * residual.  D must be 128 (PLX_ERR_UNSUPPORTED otherwise); PLX_ERR_BAD_SHAPE if a scale is not a
+ * residual.  D in {64, 128} (at D = 64 the rows are 64 bytes: the compute-matched shape of Sec. 3.3
+ * "Profiling Result"); groups above four heads per KV head are served by several CTAs of at most four.
+ * PLX_ERR_BAD_SHAPE if a scale is not a
  * positive finite number.
  */
 int parallax_decode_fwd_fp8(const void* q, const void* r, const void* k_cache, const void* v_cache,
@@ -363,7 +365,7 @@ int parallax_decode_fwd_multi_paged(const void* q, const void* r, const void* k_
  *   k_cache, v_cache   contiguous [B, Hkv, T_max, D] (block_table NULL), or page pools
  *                      [num_pages, Hkv, page_size, D] with block_table [B, max_pages_per_seq]
  *                      (then T_max is ignored: the capacity is page_size * max_pages_per_seq)
- *   kv_dtype           PLX_KV_BF16 or PLX_KV_E4M3 (D = 128 only); for e4m3 either the scalars k_scale,
+ *   kv_dtype           PLX_KV_BF16 or PLX_KV_E4M3; for e4m3 either the scalars k_scale,
  *                      v_scale or the device arrays k_scales, v_scales [Hkv] (both non-NULL)
  *   seqlens, scale, out_dtype, workspace, workspace_bytes, num_splits, stream: as parallax_decode_fwd_ex
  *                      (workspace sized for Hq * Lq query heads)

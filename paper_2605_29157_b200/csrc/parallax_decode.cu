@@ -370,8 +370,10 @@ __device__ __forceinline__ void merge_row(const float* __restrict__ base, int co
 // ---------------------------------------------------------------------------
 template <int D, int NSTAGES, bool FP8 = false>
 struct SmemLayout {
-    static constexpr int kHalves = FP8 ? D / 128 : D / 64;    // 128-byte column blocks per row
-    static constexpr int kHalfBytes = kTileKeys * 128;        // one swizzled [16 x 64] bf16 box
+    static constexpr int kRowBytes = FP8 ? D : 2 * D;         // bytes of one cache row
+    static constexpr int kBoxBytes = kRowBytes < 128 ? kRowBytes : 128;  // bytes of a row inside one TMA box
+    static constexpr int kHalves = kRowBytes / kBoxBytes;     // column blocks (TMA boxes) per row
+    static constexpr int kHalfBytes = kTileKeys * kBoxBytes;  // one swizzled [16 keys x 128 (64) bytes] box
     static constexpr int kTensorBytes = kHalves * kHalfBytes; // K (or V) tile
     static constexpr int kStageBytes = 2 * kTensorBytes;      // K tile then V tile
     static constexpr int kRingBytes = kWarps * NSTAGES * kStageBytes;
@@ -389,8 +391,18 @@ __global__ void __launch_bounds__(kThreads, CTAS)
 plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                   const KernelParams p)
 {
-    static_assert(!FP8 || D == 128, "the fp8 cache variant is built for 128-byte rows");
+    static_assert(SmemLayout<D, NSTAGES, FP8>::kBoxBytes == 128 || (FP8 && D == 64), "64-byte rows: the e4m3 cache at D = 64");
     using SL = SmemLayout<D, NSTAGES, FP8>;
+    // Byte offset of 16-byte chunk `chunk` of row `row` inside a K or V tile.  128-byte boxes use the 128-byte
+    // swizzle (chunk index XOR row mod 8); the 64-byte rows of an e4m3 cache at D = 64 use the 64-byte swizzle
+    // (chunk index XOR (row / 2) mod 4).  Eight consecutive rows of one chunk fall into eight different
+    // 16-byte bank groups either way.
+    auto tile_off = [](int row, int chunk) -> uint32_t {
+        if constexpr (SL::kBoxBytes == 128)
+            return static_cast<uint32_t>((chunk >> 3) * SL::kHalfBytes + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
+        else
+            return static_cast<uint32_t>(row * 64 + ((chunk ^ ((row >> 1) & 3)) << 4));
+    };
     // lazy-rescale threshold in log2 units: the weights reach the value product as fp16 in the FP8
     // variant, so they are kept below 2^4 (P2 = P1 * S2 must stay inside the fp16 range)
     constexpr float kThreshold = FP8 ? 4.0f : kRescaleThreshold;
@@ -630,10 +642,11 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             // Rows past the context may hold anything (NaN included): clear them in shared memory
             // so they contribute exact zeros to both products.
             uint8_t* tile = smem + (sK - base_addr);
-            for (int i = lane; i < 2 * SL::kHalves * 128; i += 32) {
-                const int box = i >> 7, rr = (i & 127) >> 3, ch = i & 7;
+            constexpr int kChunksPerBoxRow = SL::kBoxBytes / 16, kChunksPerBox = kTileKeys * kChunksPerBoxRow;
+            for (int i = lane; i < 2 * SL::kHalves * kChunksPerBox; i += 32) {  // every 16-byte chunk of the K and the V tile
+                const int box = i / kChunksPerBox, rr = (i % kChunksPerBox) / kChunksPerBoxRow, ch = i % kChunksPerBoxRow;
                 if (rr >= valid)
-                    *reinterpret_cast<uint4*>(tile + box * SL::kHalfBytes + rr * 128 + ch * 16) =
+                    *reinterpret_cast<uint4*>(tile + box * SL::kHalfBytes + rr * SL::kBoxBytes + ch * 16) =
                         make_uint4(0u, 0u, 0u, 0u);
             }
             __syncwarp();
@@ -651,7 +664,7 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             for (int kq = 0; kq < D / 32; ++kq) {  // one ldmatrix covers 16 keys x 32 dimensions = two k-steps
                 const int chunk = kq * 2 + k_csel;
                 uint32_t a[4];
-                ldmatrix_x4(a, sK + k_row * 128 + (((chunk & 7) ^ (k_row & 7)) << 4));
+                ldmatrix_x4(a, sK + tile_off(k_row, chunk));
                 const uint32_t f0[4] = {e4m3x2_to_f16x2(a[0], false), e4m3x2_to_f16x2(a[1], false),
                                         e4m3x2_to_f16x2(a[0], true), e4m3x2_to_f16x2(a[1], true)};
                 const uint32_t f1[4] = {e4m3x2_to_f16x2(a[2], false), e4m3x2_to_f16x2(a[3], false),
@@ -667,7 +680,7 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             for (int ks = 0; ks < KSTEPS; ++ks) {
                 const int chunk = ks * 2 + k_csel;
                 uint32_t a[4];
-                ldmatrix_x4(a, sK + (chunk >> 3) * SL::kHalfBytes + k_row * 128 + (((chunk & 7) ^ (k_row & 7)) << 4));
+                ldmatrix_x4(a, sK + tile_off(k_row, chunk));
 #pragma unroll
                 for (int qd = 0; qd < NQ; ++qd) mma_bf16((ks & 1) ? c2[qd] : c[qd], a, bqr[qd][ks][0], bqr[qd][ks][1]);
             }
@@ -816,7 +829,7 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             for (int mq = 0; mq < D / 32; ++mq) {  // one transposed ldmatrix covers two 16-dimension m-tiles
                 const int chunk = mq * 2 + v_csel;
                 uint32_t a[4];
-                ldmatrix_x4_trans(a, sV + v_row * 128 + (((chunk & 7) ^ (v_row & 7)) << 4));
+                ldmatrix_x4_trans(a, sV + tile_off(v_row, chunk));
                 // a register holds (key 2t: dims 2g, 2g+1 | key 2t+1: dims 2g, 2g+1): regroup by dimension
                 uint32_t x[4];
 #pragma unroll
@@ -844,8 +857,8 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             for (int mt = 0; mt < MTILES; mt += 2) {  // two m-tiles at a time: the residual MMAs follow two others
                 uint32_t a0[4], a1[4];
                 const int ch0 = mt * 2 + v_csel, ch1 = ch0 + 2;
-                ldmatrix_x4_trans(a0, sV + (ch0 >> 3) * SL::kHalfBytes + v_row * 128 + (((ch0 & 7) ^ (v_row & 7)) << 4));
-                ldmatrix_x4_trans(a1, sV + (ch1 >> 3) * SL::kHalfBytes + v_row * 128 + (((ch1 & 7) ^ (v_row & 7)) << 4));
+                ldmatrix_x4_trans(a0, sV + tile_off(v_row, ch0));
+                ldmatrix_x4_trans(a1, sV + tile_off(v_row, ch1));
 #pragma unroll
                 for (int qd = 0; qd < NQ; ++qd) {
                     mma_bf16(o[qd][mt], a0, pb0[qd], pb1[qd]);
@@ -1295,19 +1308,27 @@ int dispatch_main(int D, int G, const CUtensorMap& tmK, const CUtensorMap& tmV, 
     if (fp8) {
         // e4m3 cache, D = 128: 4 KiB stages, the byte geometry of a 16-bit cache at D = 64, and the same
         // measured optimum: four CTAs per SM (128 registers per thread at G <= 2), two stages per warp
-        // when the grid fills the device, three otherwise.  G = 4 needs ~210 registers: two CTAs per SM.
-        if (D != 128) return PLX_ERR_UNSUPPORTED;
+        // when the grid fills the device, three otherwise.  G = 3, 4 need ~155 registers: two CTAs per SM.
+        // D = 64: 64-byte rows, 2 KiB stages (the compute-matched shape of Sec. 3.3 over an e4m3 cache).
         int num_sms = 0;
         if (int rc = device_sm_count(&num_sms); rc != PLX_OK) return rc;
         const long long n_ctas = static_cast<long long>(kp.B) * kp.Hkv * kp.num_splits;
-        if (kp.chunk_len <= 2 * kChunkGranule || n_ctas >= 3LL * num_sms) {
-            if (G == 1) return launch_main<128, 1, 2, kCtasPerSmFp8, true>(tmK, tmV, kp, stream);
-            if (G == 2) return launch_main<128, 2, 2, kCtasPerSmFp8, true>(tmK, tmV, kp, stream);
+        const bool two_stage = kp.chunk_len <= 2 * kChunkGranule || n_ctas >= 3LL * num_sms;
+        if (D == 128) {
+            if (two_stage) {
+                if (G == 1) return launch_main<128, 1, 2, kCtasPerSmFp8, true>(tmK, tmV, kp, stream);
+                if (G == 2) return launch_main<128, 2, 2, kCtasPerSmFp8, true>(tmK, tmV, kp, stream);
+            }
+            if (G == 1) return launch_main<128, 1, PLX_STAGES_FP8, kCtasPerSmFp8, true>(tmK, tmV, kp, stream);
+            if (G == 2) return launch_main<128, 2, PLX_STAGES_FP8, kCtasPerSmFp8, true>(tmK, tmV, kp, stream);
+            if (G == 3) return launch_main<128, 3, PLX_STAGES_FP8, 2, true>(tmK, tmV, kp, stream);
+            if (G == 4) return launch_main<128, 4, PLX_STAGES_FP8, 2, true>(tmK, tmV, kp, stream);
+        } else if (D == 64) {
+            if (G == 1) return launch_main<64, 1, PLX_STAGES_FP8, kCtasPerSmFp8, true>(tmK, tmV, kp, stream);
+            if (G == 2) return launch_main<64, 2, PLX_STAGES_FP8, kCtasPerSmFp8, true>(tmK, tmV, kp, stream);
+            if (G == 3) return launch_main<64, 3, PLX_STAGES_FP8, kCtasPerSmFp8, true>(tmK, tmV, kp, stream);
+            if (G == 4) return launch_main<64, 4, PLX_STAGES_FP8, kCtasPerSmFp8, true>(tmK, tmV, kp, stream);
         }
-        if (G == 1) return launch_main<128, 1, PLX_STAGES_FP8, kCtasPerSmFp8, true>(tmK, tmV, kp, stream);
-        if (G == 2) return launch_main<128, 2, PLX_STAGES_FP8, kCtasPerSmFp8, true>(tmK, tmV, kp, stream);
-        if (G == 3) return launch_main<128, 3, PLX_STAGES_FP8, 2, true>(tmK, tmV, kp, stream);
-        if (G == 4) return launch_main<128, 4, PLX_STAGES_FP8, 2, true>(tmK, tmV, kp, stream);
         return PLX_ERR_UNSUPPORTED;
     }
     // D = 128: 8 KiB stages, three per warp, two CTAs per SM (192 KiB of K/V in flight per SM).  A chunk
@@ -1539,7 +1560,6 @@ static int decode_fwd_impl(const void* q, const void* r, const void* k_cache, co
 {
     int rc = check_inputs(q, r, k_cache, v_cache, B, Hq, Hkv, D, T_max);
     if (rc != PLX_OK) return rc;
-    if (fp8 && D != 128) return PLX_ERR_UNSUPPORTED;
     if (!out) return PLX_ERR_NULL_POINTER;
     if (out_dtype != PLX_OUT_BF16 && out_dtype != PLX_OUT_F32) return PLX_ERR_BAD_SHAPE;
     if (num_splits < 0 || num_splits > PLX_MAX_SPLITS) return PLX_ERR_BAD_SHAPE;

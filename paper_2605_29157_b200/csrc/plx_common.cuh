@@ -134,8 +134,8 @@ inline EncodeTiledFn get_encode_fn()
     return fn;
 }
 
-// bf16 [rows, D] row-major viewed in boxes of [box_rows rows, 64 columns] with the 128-byte swizzle;
-// rows past the end read as zero.  Encoding costs about a microsecond of host time and the result is
+// bf16 [rows, D] row-major viewed in boxes of [box_rows rows, 64 columns] with the 128-byte swizzle (rows of
+// 32 columns = 64 bytes: boxes of [box_rows rows, 32 columns] with the 64-byte swizzle); rows past the end read as zero.  Encoding costs about a microsecond of host time and the result is
 // a pure function of the arguments, so the last encodings are kept in a small direct-mapped cache
 // (decode calls are launch-bound on small batches and reuse the same caches step after step).
 inline int make_tensor_map_2d(CUtensorMap* tm, const void* base, int D, uint64_t rows, uint32_t box_rows,
@@ -166,10 +166,11 @@ inline int make_tensor_map_2d(CUtensorMap* tm, const void* base, int D, uint64_t
     if (!enc) return PLX_ERR_CUDA;
     const cuuint64_t dims[2] = {static_cast<cuuint64_t>(D), rows};
     const cuuint64_t strides[1] = {static_cast<cuuint64_t>(D) * 2};
-    const cuuint32_t box[2] = {64, box_rows};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(D < 64 ? D : 64), box_rows};
     const cuuint32_t estr[2] = {1, 1};
+    const CUtensorMapSwizzle swizzle = D < 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B;
     CUresult rc = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, promotion,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, promotion,
                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (rc == CUDA_ERROR_INVALID_CONTEXT || rc == CUDA_ERROR_NOT_INITIALIZED) {
         // The encoder is a driver call and needs a current context; a host thread that has made no runtime
@@ -178,7 +179,7 @@ inline int make_tensor_map_2d(CUtensorMap* tm, const void* base, int D, uint64_t
         // has a context already.
         if (cudaFree(nullptr) != cudaSuccess) return PLX_ERR_CUDA;
         rc = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, promotion,
+                 CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, promotion,
                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     }
     if (rc != CUDA_SUCCESS) return PLX_ERR_CUDA;

@@ -39,19 +39,43 @@ def run_case(plx, oracle, cfg, out_dtype=torch.float32, num_splits=0, poison=Fal
     return assert_parity(out.float().cpu().numpy(), want, out_dtype, cfg.name)
 
 
+@pytest.mark.parametrize("D", [128, 64])
 @pytest.mark.parametrize("G", [1, 2, 3, 4])
 @pytest.mark.parametrize("T", [1, 2, 15, 16, 17, 63, 64, 65, 127, 300, 1000])
-def test_fp8_shape_sweep_single_split(plx, oracle, G, T):
-    cfg = wl.DecodeConfig(f"fp8 G={G} T={T}", B=2, Hq=2 * G, Hkv=2, D=128, T_max=T, seed=900 + T)
+def test_fp8_shape_sweep_single_split(plx, oracle, D, G, T):
+    """D = 64: 64-byte cache rows, staged in boxes with the 64-byte swizzle."""
+    cfg = wl.DecodeConfig(f"fp8 D={D} G={G} T={T}", B=2, Hq=2 * G, Hkv=2, D=D, T_max=T, seed=900 + T)
     run_case(plx, oracle, cfg, num_splits=1)
 
 
-@pytest.mark.parametrize("G", [1, 2, 4])
+@pytest.mark.parametrize("D,G", [(128, 1), (128, 2), (128, 4), (64, 2), (64, 3)])
 @pytest.mark.parametrize("T,ns", [(130, 2), (1000, 3), (4096, 0), (5000, 7), (12800, 120)])
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
-def test_fp8_split_kv(plx, oracle, G, T, ns, out_dtype):
-    cfg = wl.DecodeConfig(f"fp8 split G={G} T={T} ns={ns}", B=3, Hq=2 * G, Hkv=2, D=128, T_max=T, seed=11 * T + ns)
+def test_fp8_split_kv(plx, oracle, D, G, T, ns, out_dtype):
+    cfg = wl.DecodeConfig(f"fp8 split D={D} G={G} T={T} ns={ns}", B=3, Hq=2 * G, Hkv=2, D=D, T_max=T, seed=11 * T + ns)
     run_case(plx, oracle, cfg, out_dtype=out_dtype, num_splits=ns)
+
+
+def test_fp8_head_dim_64_ragged_paged_and_groups_above_four(plx, oracle):
+    """The compute-matched shape over an e4m3 cache: ragged lengths with NaN padding, a paged cache, and a
+    group of eight query heads (two CTAs of four per KV head in this variant)."""
+    cfg = wl.DecodeConfig("fp8 d64 ragged", B=5, Hq=16, Hkv=2, D=64, T_max=2500, ragged=(1, 2500), seed=955)
+    run_case(plx, oracle, cfg, poison=True)
+    x = wl.make_inputs(cfg, "cuda", poison_padding=True)
+    k8, ks = wl.quantize_e4m3(x["k"])
+    v8, vs = wl.quantize_e4m3(x["v"])
+    ks32, vs32 = float(np.float32(ks)), float(np.float32(vs))
+    kp, vp, table = wl.to_paged(k8.to(torch.float16), v8.to(torch.float16), 64, seed=3)   # fp16 holds every e4m3 value and NaN
+    kp, vp = kp.to(torch.float8_e4m3fn), vp.to(torch.float8_e4m3fn)
+    ws = plx.alloc_workspace(cfg.B, cfg.Hq, cfg.D, plx.PLX_MAX_SPLITS, "cuda")
+    ref = torch.empty(cfg.B, cfg.Hq, cfg.D, dtype=torch.float32, device="cuda")
+    got = torch.full_like(ref, float("nan"))
+    plx.parallax_decode_fwd_fp8(x["q"], x["r"], k8, v8, x["seqlens"], ref, cfg.scale, ks32, vs32, ws, 3)
+    plx.parallax_decode_fwd_paged_fp8(x["q"], x["r"], kp, vp, table, x["seqlens"], got, cfg.scale, ks32, vs32, ws, 3)
+    torch.cuda.synchronize()
+    assert plx.parallax_workspace_status(ws) == 0
+    # same arithmetic, but the padded paged context is cut into other chunks: equal up to fp32 summation order
+    assert torch.isfinite(got).all() and (got - ref).abs().max().item() <= 1e-4 * ref.abs().max().item()
 
 
 def test_fp8_ragged_batch_with_poisoned_padding(plx, oracle):
@@ -81,10 +105,10 @@ def test_fp8_large_probe(plx, oracle):
 
 
 def test_fp8_rejects_other_head_dims_and_bad_scales(plx):
-    cfg = wl.DecodeConfig("fp8 d64", B=1, Hq=2, Hkv=1, D=64, T_max=64, seed=1)
+    cfg = wl.DecodeConfig("fp8 d32", B=1, Hq=2, Hkv=1, D=32, T_max=64, seed=1)
     x = wl.make_inputs(cfg, "cuda")
     k8, _ = wl.quantize_e4m3(x["k"])
-    out = torch.empty(1, 2, 64, dtype=torch.float32, device="cuda")
+    out = torch.empty(1, 2, 32, dtype=torch.float32, device="cuda")
     with pytest.raises(plx.ParallaxError) as e:
         plx.parallax_decode_fwd_fp8(x["q"], x["r"], k8, k8, None, out, 0.1, 1.0, 1.0, None, 1)
     assert e.value.status == plx.PLX_ERR_UNSUPPORTED

@@ -169,7 +169,7 @@ def test_serving_variant_entry_points_validate_on_the_host(lib):
     def fp8(D=128, ks=0.5, vs=0.5, k=fake):
         return L.parallax_decode_fwd_fp8(fake, fake, k, fake, none, fake, 2, 4, 2, D, 64, 0.1, ks, vs, 0, none, 0, 1, none)
 
-    assert fp8(D=64) == lib.PLX_ERR_UNSUPPORTED
+    assert fp8(D=96) == lib.PLX_ERR_UNSUPPORTED
     assert fp8(ks=0.0) == lib.PLX_ERR_BAD_SHAPE
     assert fp8(vs=float("inf")) == lib.PLX_ERR_BAD_SHAPE
     assert fp8(vs=float("nan")) == lib.PLX_ERR_BAD_SHAPE
@@ -222,7 +222,7 @@ def test_per_head_scale_and_one_call_step_entry_points_validate_on_the_host(lib)
     assert per_head(ks=none) == lib.PLX_ERR_NULL_POINTER
     assert per_head(vs=none) == lib.PLX_ERR_NULL_POINTER
     assert per_head(ks=odd) == lib.PLX_ERR_ALIGNMENT
-    assert per_head(D=64) == lib.PLX_ERR_UNSUPPORTED
+    assert per_head(D=96) == lib.PLX_ERR_UNSUPPORTED
     assert per_head(Hq=5) == lib.PLX_ERR_BAD_SHAPE
 
     def paged_per_head(table=fake, ks=fake, ps=64):
