@@ -569,14 +569,20 @@ def quick_config(name, sampler, read_peak=None, steps=20, warmup=5):
 def quick_tensor_workload(name, local_rank=0):
     """Short run of a tensor-core workload (multi-token forward or backward) for the default line: value,
     roofline fraction against the sustained bf16 peak, clocks."""
-    ns = argparse.Namespace(workload=name, steps=5, warmup=3, batch=0, kv_sets=0, plain_bf16_p=False,
-                            no_cpu_baseline=True, cpu_seconds=0.0)
-    runner = run_prefill if name in wl.PREFILL_CONFIGS else run_backward
-    r = runner(ns, 0, 1, local_rank)
-    torch.cuda.empty_cache()
-    return {"metric": r["metric"], "value": r["value"], "unit": r["unit"], "ms_per_step": r["ms_per_step"],
-            "roofline_frac_of_sustained_bf16": r["roofline"]["frac"], "roofline_kernel": r["roofline"]["kernel"],
-            "workload": r["config"]["workload"], "clocks": r["clocks"], **r["timing"]}
+    def one(mode):
+        ns = argparse.Namespace(workload=name, steps=5, warmup=3, batch=0, kv_sets=0, plain_bf16_p=False, p_precision=mode,
+                                no_cpu_baseline=True, cpu_seconds=0.0)
+        runner = run_prefill if name in wl.PREFILL_CONFIGS else run_backward
+        r = runner(ns, 0, 1, local_rank)
+        torch.cuda.empty_cache()
+        return {"metric": r["metric"], "value": r["value"], "unit": r["unit"], "ms_per_step": r["ms_per_step"],
+                "roofline_frac_of_sustained_bf16": r["roofline"]["frac"], "roofline_kernel": r["roofline"]["kernel"],
+                "workload": r["config"]["workload"], "clocks": r["clocks"], **r["timing"]}
+    res = one("residual")
+    if name in wl.PREFILL_CONFIGS:   # the same workload with residual products only where rows see few keys
+        res["p_precision"] = "bf16+residual"
+        res["adaptive_p_precision"] = one("adaptive")
+    return res
 
 
 def single_thread_oracle_c2():
@@ -606,8 +612,17 @@ def run_prefill(args, rank, world, local_rank):
     nsets = args.kv_sets or 2
     sets = [wl.make_prefill_inputs(wl.scaled(cfg, seed=cfg.seed + 17 * i), Lq, dev) for i in range(nsets)]
     flops = wl.prefill_flops(cfg, Lq)
-    prec = plx.PLX_P_BF16 if args.plain_bf16_p else plx.PLX_P_BF16_RESIDUAL
-    mma_factor = 1.0 if args.plain_bf16_p else 1.5
+    mode = "plain" if args.plain_bf16_p else getattr(args, "p_precision", "residual")
+    prec = {"plain": plx.PLX_P_BF16, "residual": plx.PLX_P_BF16_RESIDUAL, "adaptive": plx.PLX_P_BF16_ADAPTIVE}[mode]
+    # executed / algorithmic tensor work: the residual products add half; in the adaptive mode only in the row
+    # tiles in which some row sees fewer than PLX_P_ADAPTIVE_MIN_KEYS keys
+    if mode == "adaptive":
+        i = np.arange(Lq, dtype=np.int64)
+        vis = np.maximum(cfg.T_max - Lq + i + 1, 0)
+        first = np.maximum(cfg.T_max - Lq + 128 * (i // 128) + 1, 0)
+        mma_factor = 1.0 + 0.5 * float(vis[first < plx.PLX_P_ADAPTIVE_MIN_KEYS].sum()) / float(vis.sum())
+    else:
+        mma_factor = 1.0 if mode == "plain" else 1.5
     out = torch.empty(cfg.B, cfg.Hq, Lq, cfg.D, dtype=torch.bfloat16, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     stream = torch.cuda.current_stream()
@@ -670,7 +685,9 @@ def run_prefill(args, rank, world, local_rank):
                      "peak_source": ("measured" if peaks else "fallback") + " cuBLAS bf16, sustained (kernel timed back to back for the whole step)",
                      "unit": "TFLOP/s", "frac": round(achieved / peak, 4), "frac_of_burst_peak": round(achieved / burst, 4),
                      "executed_tflops_incl_residual_mmas": round(achieved * mma_factor, 1),
-                     "p_precision": "bf16" if args.plain_bf16_p else "bf16+residual",
+                     "p_precision": {"plain": "bf16", "residual": "bf16+residual",
+                                     "adaptive": f"bf16+residual in row tiles with a row of fewer than {plx.PLX_P_ADAPTIVE_MIN_KEYS} "
+                                                 "keys, plain bf16 elsewhere"}[mode],
                      "algorithmic_flops_per_launch": flops,
                      "traffic": None if args.batch else ncu_traffic(cfg.name)[0],
                      "traffic_source": None if args.batch else ncu_traffic(cfg.name)[1]},
@@ -1044,6 +1061,8 @@ def main(argv=None):
     ap.add_argument("--kv-sets", type=int, default=0, help="number of KV cache sets rotated between steps")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (profiling captures on a smaller case)")
     ap.add_argument("--plain-bf16-p", action="store_true", help="prefill workloads: PLX_P_BF16 (no residual tiles)")
+    ap.add_argument("--p-precision", default="residual", choices=["residual", "adaptive", "plain"],
+                    help="prefill workloads: precision of the softmax weights on their way into the value product")
     ap.add_argument("--new-tokens", type=int, default=1,
                     help="decode workloads: this many new tokens per sequence and step (parallax_decode_fwd_multi)")
     ap.add_argument("--page-size", type=int, default=0, help="decode workloads: run over a paged KV cache with this page size")

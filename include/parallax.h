@@ -70,6 +70,13 @@ extern "C" {
 /* Precision of the softmax weights P1, P2 on their way into the value product (prefill entry point). */
 #define PLX_P_BF16_RESIDUAL 0 /* bf16 plus its bf16 rounding residual: fp32-class result (default) */
 #define PLX_P_BF16 1          /* plain bf16: faster, relative error ~2^-9 * sqrt(D) on rows with few keys */
+/* residuals only in the 128-row tiles in which some row sees fewer than PLX_P_ADAPTIVE_MIN_KEYS keys, plain
+ * bf16 weights elsewhere: the few-key rows (where the two branches' cancellation amplifies the weights'
+ * rounding) keep the fp32-class result, rows that average over a thousand keys or more get the precision of a
+ * bf16 tensor-core attention kernel (relative RMS error ~1.6e-3, the level of a bf16 output's own rounding),
+ * and a long prefill executes about 1.03 instead of 1.5 times its algorithmic tensor work */
+#define PLX_P_BF16_ADAPTIVE 2
+#define PLX_P_ADAPTIVE_MIN_KEYS 1024
 
 /* Largest split count any entry point accepts. */
 #define PLX_MAX_SPLITS 1024

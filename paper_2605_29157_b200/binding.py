@@ -33,6 +33,8 @@ PLX_OUT_BF16 = 0
 PLX_OUT_F32 = 1
 PLX_P_BF16_RESIDUAL = 0
 PLX_P_BF16 = 1
+PLX_P_BF16_ADAPTIVE = 2
+PLX_P_ADAPTIVE_MIN_KEYS = 1024
 PLX_MAX_SPLITS = 1024
 
 # PARALLAX_LIBRARY selects another build of the same library (the index-checking debug build,

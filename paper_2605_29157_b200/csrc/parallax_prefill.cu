@@ -114,6 +114,11 @@ struct PrefillParams {
     // finished by the decode path's merge kernel.  partials == nullptr: one CTA per tile, final output.
     float* partials;
     int num_splits, tiles_per_split;
+    // PLX_P_BF16_ADAPTIVE runs as two launches over the same tiles, the plain build and the residual build; a
+    // CTA leaves at once unless its tile is of its launch's kind: tile_filter 1 = only row tiles in which some
+    // row sees fewer than residual_min_keys keys, 2 = only the others, 0 = every tile.  qt_hi: one past the last
+    // row tile this launch covers (the host narrows the grids when the contexts are uniform).
+    int tile_filter, residual_min_keys, qt_hi;
 };
 
 // barrier among the softmax warps only (named barrier 1)
@@ -158,7 +163,7 @@ plx_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     const int heads = p.B * (pack > 1 ? p.Hkv : p.Hq);  // tiles' owners: KV heads when packed, else query heads
     const int split = p.partials ? static_cast<int>(blockIdx.x % p.num_splits) : 0;
     const int tile_id = p.partials ? static_cast<int>(blockIdx.x / p.num_splits) : static_cast<int>(blockIdx.x);
-    const int qt = p.q_tiles - 1 - tile_id / heads;  // heaviest (latest) tiles first
+    const int qt = p.qt_hi - 1 - tile_id / heads;  // heaviest (latest) tiles first
     const int bh = tile_id % heads;
     int b, hq, hkv;
     if (pack > 1) {
@@ -175,6 +180,11 @@ plx_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     int L = p.seqlens ? p.seqlens[b] : p.T_max;
     L = max(0, min(L, p.T_max));
     const int q0 = qt * BM;
+    if (p.tile_filter) {
+        // fewest keys a row of this tile sees (a packed tile holds token 0 of every head)
+        const bool few = L - p.Lq + (pack > 1 ? 0 : q0) + 1 < p.residual_min_keys;
+        if (few != (p.tile_filter == 1)) return;
+    }
     const int q_hi = min(q0 + BM, rows);
     const int tok_hi = pack > 1 ? p.Lq : q_hi;                 // one past the latest token in this tile
     const int kv_end = min(L, max(0, L - p.Lq + tok_hi));  // keys visible to the latest token of this tile
@@ -663,7 +673,8 @@ static int prefill_impl(const void* q, const void* r, const void* k_cache, const
                         int max_pages = 0, long long pool_rows = 0, void* workspace = nullptr,
                         size_t workspace_bytes = 0, int num_splits = 1)
 {
-    if (p_precision != PLX_P_BF16_RESIDUAL && p_precision != PLX_P_BF16) return PLX_ERR_BAD_SHAPE;
+    if (p_precision != PLX_P_BF16_RESIDUAL && p_precision != PLX_P_BF16 && p_precision != PLX_P_BF16_ADAPTIVE)
+        return PLX_ERR_BAD_SHAPE;
     if (!q || !r || !k_cache || !v_cache || !out) return PLX_ERR_NULL_POINTER;
     if (B <= 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || Lq <= 0 || T_max <= 0 || Hq % Hkv != 0) return PLX_ERR_BAD_SHAPE;
     if (D != 64 && D != 128) return PLX_ERR_UNSUPPORTED;
@@ -728,22 +739,51 @@ static int prefill_impl(const void* q, const void* r, const void* k_cache, const
     ns = (tiles_max + tps - 1) / tps;  // no split without a tile
     PrefillParams pp{seqlens, out, status, B, Hq, Hkv, Lq, T_max, q_tiles, scale * 1.4426950408889634f, out_dtype,
                      lse, tbar, vbar, block_table, page_size, max_pages, pack,
-                     ns > 1 ? static_cast<float*>(workspace) : nullptr, ns, tps};
+                     ns > 1 ? static_cast<float*>(workspace) : nullptr, ns, tps, 0, 0, q_tiles};
     if (base_ctas * ns > 0x7fffffffLL) return PLX_ERR_BAD_SHAPE;
-    const unsigned grid = static_cast<unsigned>(base_ctas * ns);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const bool res = p_precision == PLX_P_BF16_RESIDUAL;
     PlxNvtxRange nvtx_range("plx_prefill_fwd");
-    if (D == 128) {
-        if (res)
-            plx_prefill_kernel<true, 128><<<grid, kPrefillThreads, kSmemBytes, st>>>(tmQ, tmR, tmK, tmV, pp);
-        else
-            plx_prefill_kernel<false, 128><<<grid, kPrefillThreads, kSmemBytes, st>>>(tmQ, tmR, tmK, tmV, pp);
+    const long long ctas_per_qt = static_cast<long long>(B) * (pack > 1 ? Hkv : Hq) * ns;
+    auto launch = [&](bool res, const PrefillParams& prm, int qt_lo, int qt_hi) {
+        if (qt_hi <= qt_lo) return;
+        PrefillParams lp = prm;
+        lp.qt_hi = qt_hi;
+        const unsigned grid = static_cast<unsigned>((qt_hi - qt_lo) * ctas_per_qt);
+        if (D == 128) {
+            if (res)
+                plx_prefill_kernel<true, 128><<<grid, kPrefillThreads, kSmemBytes, st>>>(tmQ, tmR, tmK, tmV, lp);
+            else
+                plx_prefill_kernel<false, 128><<<grid, kPrefillThreads, kSmemBytes, st>>>(tmQ, tmR, tmK, tmV, lp);
+        } else {
+            if (res)
+                plx_prefill_kernel<true, 64><<<grid, kPrefillThreads, kSmemBytes, st>>>(tmQ, tmR, tmK, tmV, lp);
+            else
+                plx_prefill_kernel<false, 64><<<grid, kPrefillThreads, kSmemBytes, st>>>(tmQ, tmR, tmK, tmV, lp);
+        }
+    };
+    if (p_precision == PLX_P_BF16_ADAPTIVE) {
+        // Two launches: the plain build for the row tiles all of whose rows see at least PLX_P_ADAPTIVE_MIN_KEYS
+        // keys, the residual build for the others.  Uniform contexts: the boundary is known here and each grid
+        // covers only its tiles; ragged contexts: both grids cover every tile and a CTA of the wrong kind leaves
+        // at once (the boundary depends on seqlens, which lives on the device).
+        pp.residual_min_keys = PLX_P_ADAPTIVE_MIN_KEYS;
+        int qt_split = 0;  // row tiles below it carry residuals
+        if (!seqlens) {
+            if (pack > 1) {
+                qt_split = (T_max - Lq + 1 < PLX_P_ADAPTIVE_MIN_KEYS) ? 1 : 0;
+            } else {
+                const long long first_plain_row = static_cast<long long>(PLX_P_ADAPTIVE_MIN_KEYS) - 1 - (T_max - Lq);  // q0 >= this: plain
+                qt_split = first_plain_row <= 0 ? 0 : static_cast<int>((first_plain_row + BM - 1) / BM);
+                if (qt_split > q_tiles) qt_split = q_tiles;
+            }
+        }
+        PrefillParams plain = pp, resid = pp;
+        plain.tile_filter = 2;
+        resid.tile_filter = 1;
+        launch(false, plain, seqlens ? 0 : qt_split, q_tiles);
+        launch(true, resid, 0, seqlens ? q_tiles : qt_split);
     } else {
-        if (res)
-            plx_prefill_kernel<true, 64><<<grid, kPrefillThreads, kSmemBytes, st>>>(tmQ, tmR, tmK, tmV, pp);
-        else
-            plx_prefill_kernel<false, 64><<<grid, kPrefillThreads, kSmemBytes, st>>>(tmQ, tmR, tmK, tmV, pp);
+        launch(p_precision == PLX_P_BF16_RESIDUAL, pp, 0, q_tiles);
     }
     if (cudaGetLastError() != cudaSuccess) return PLX_ERR_CUDA;
     if (ns > 1)  // finish the rows: the decode path's merge over B * Hq * Lq rows of ns records each

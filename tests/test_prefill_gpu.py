@@ -107,6 +107,37 @@ def test_prefill_plain_bf16_weights(plx, oracle):
     assert e["max_abs"] <= MAX_ABS_TOL and e["mean_abs"] <= MEAN_ABS_TOL and e["rel_rms"] <= 1e-2, e
 
 
+@pytest.mark.parametrize("D,G,Lq,T", [(128, 2, 2500, 2500), (64, 2, 2400, 2400), (128, 1, 700, 1900), (128, 4, 16, 3000),
+                                      (128, 4, 20, 600)])
+def test_prefill_adaptive_residuals(plx, oracle, D, G, Lq, T):
+    """PLX_P_BF16_ADAPTIVE: row tiles in which some row sees fewer than PLX_P_ADAPTIVE_MIN_KEYS keys carry the
+    residual products and keep the fp32-class result; the other tiles send plain bf16 weights, whose rounding
+    then averages over at least that many keys: the stated bars hold with room, the relative RMS error is at
+    the level of a bf16 output's own rounding.  Covers both tile kinds in one call, a chunk whose rows all see
+    more than the limit (every tile plain, incl. the two-buffer use of the P region), and a packed tile."""
+    cfg = wl.DecodeConfig("adaptive", B=2, Hq=2 * G, Hkv=2, D=D, T_max=T, seed=350 + Lq)
+    x = wl.make_prefill_inputs(cfg, Lq, "cuda")
+    out = torch.full((cfg.B, cfg.Hq, Lq, cfg.D), float("nan"), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    plx.parallax_prefill_fwd(x["q"], x["r"], x["k"], x["v"], None, out, cfg.scale, status, p_precision=plx.PLX_P_BF16_ADAPTIVE)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    bits = {n: wl.bf16_bits(x[n]) for n in ("q", "r", "k", "v")}
+    want, _ = oracle.prefill_bf16(bits["q"], bits["r"], bits["k"], bits["v"], None, cfg.scale)
+    got = out.cpu().numpy()
+    assert np.isfinite(got).all()
+    packed = G > 1 and G * Lq <= 128
+    first_visible = (T - Lq + 1) + (np.zeros(Lq, dtype=np.int64) if packed else 128 * (np.arange(Lq) // 128))   # fewest keys seen in the row's tile
+    with_res = first_visible < plx.PLX_P_ADAPTIVE_MIN_KEYS
+    if with_res.any():
+        e = errors(got[:, :, with_res], want[:, :, with_res])
+        assert e["max_abs"] <= MAX_ABS_TOL and e["mean_abs"] <= MEAN_ABS_TOL and e["rel_rms"] <= REL_RMS_TOL_F32, ("residual tiles", e)
+    if (~with_res).any():
+        e = errors(got[:, :, ~with_res], want[:, :, ~with_res])
+        assert e["max_abs"] <= MAX_ABS_TOL and e["mean_abs"] <= MEAN_ABS_TOL and e["rel_rms"] <= REL_RMS_TOL_BF16, ("plain tiles", e)
+        assert e["rel_rms"] > REL_RMS_TOL_F32, "these tiles were expected to run without residual products"
+
+
 @pytest.mark.parametrize("name", ["P1", "P2", "P3", "P4"])
 def test_prefill_full_size_in_the_bench_configuration(plx, oracle, name):
     """Full-size prefill workloads with the entry point, workspace and dtypes the bench times (bf16 output;
@@ -273,3 +304,37 @@ def test_prefill_paged_cache_split_kv(plx, oracle, page_size, Lq, T, ns):
     want, _ = oracle.prefill_bf16(bits["q"], bits["r"], bits["k"], bits["v"], x["seqlens_host"], cfg.scale)
     e = errors(out.cpu().numpy(), want)
     assert e["max_abs"] <= MAX_ABS_TOL and e["mean_abs"] <= MEAN_ABS_TOL and e["rel_rms"] <= REL_RMS_TOL_F32, e
+
+
+def test_prefill_adaptive_residuals_ragged_contexts(plx, oracle):
+    """Ragged contexts: which tiles carry residuals depends on seqlens (device data), so both launches of the
+    adaptive mode cover every tile and each CTA decides for itself.  Every row is written exactly once: the
+    output starts as NaN and must come back finite and within the bars of its tile's kind; split-KV too."""
+    cfg = wl.DecodeConfig("adaptive ragged", B=4, Hq=4, Hkv=2, D=128, T_max=2600, seed=377)
+    Lq = 300
+    lens = np.array([2600, 1200, 310, 0], dtype=np.int32)
+    x = wl.make_prefill_inputs(cfg, Lq, "cuda")
+    x["seqlens"] = torch.from_numpy(lens).cuda()
+    for b in range(cfg.B):
+        x["k"][b, :, int(lens[b]):] = float("nan")
+        x["v"][b, :, int(lens[b]):] = float("nan")
+    bits = {n: wl.bf16_bits(x[n]) for n in ("q", "r", "k", "v")}
+    want, _ = oracle.prefill_bf16(bits["q"], bits["r"], bits["k"], bits["v"], lens, cfg.scale)
+    ws = torch.empty(plx.parallax_prefill_workspace_bytes(cfg.B, cfg.Hq, cfg.D, Lq, 8), dtype=torch.uint8, device="cuda")
+    for ns in (1, 5):
+        out = torch.full((cfg.B, cfg.Hq, Lq, cfg.D), float("nan"), dtype=torch.float32, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        plx.parallax_prefill_fwd_ex(x["q"], x["r"], x["k"], x["v"], x["seqlens"], out, cfg.scale, ws, ns, status,
+                                    p_precision=plx.PLX_P_BF16_ADAPTIVE)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        got = out.cpu().numpy()
+        assert np.isfinite(got).all()
+        for b in range(cfg.B):
+            first_visible = (int(lens[b]) - Lq + 1) + 128 * (np.arange(Lq) // 128)
+            with_res = first_visible < plx.PLX_P_ADAPTIVE_MIN_KEYS
+            for sel, tol in ((with_res, REL_RMS_TOL_F32), (~with_res, REL_RMS_TOL_BF16)):
+                if sel.any() and np.abs(want[b][:, sel]).max() > 0:
+                    e = errors(got[b][:, sel], want[b][:, sel])
+                    assert e["max_abs"] <= MAX_ABS_TOL and e["mean_abs"] <= MEAN_ABS_TOL and e["rel_rms"] <= tol, (ns, b, e)
+        assert np.all(got[3] == 0.0)      # the empty context
