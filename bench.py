@@ -52,11 +52,13 @@ MAX_BLOCKS = 4000
 # in proportion to the batch).  An entry goes stale when its kernel changes; the bench line carries the
 # provenance string beside the number.
 NCU_TRAFFIC = {
-    "C2": (134_600_000, "plx_decode_kernel<128,2,3,2>, full-size capture (cache sets rotated, so reads miss L2)"),
-    "C3": (2_155_300_000, "plx_decode_kernel<128,2,3,2>, capture at B=32 scaled x2"),
-    "C4": (1_077_300_000, "plx_decode_kernel<128,2,3,2>, full-size capture"),
-    "C6": (2 * 541_600_000, "plx_decode_kernel<64,2,2,4>, capture at B=32 scaled x2"),
-    "P1": (8 * 51_000_000, "plx_prefill_kernel<128>, capture at B=1 scaled x8"),
+    "C2": (134_500_000, "plx_decode_kernel<128,2,3,2,0>, full-size capture (cache sets rotated, so reads miss L2)"),
+    "C3": (2_157_500_000, "plx_decode_kernel<128,2,3,2,0>, capture at B=32 scaled x2"),
+    "C4": (1_077_300_000, "plx_decode_kernel<128,2,3,2,0>, full-size capture (before the prologue was split around the "
+                          "dependency wait; byte counts unaffected)"),
+    "C5": (7_661_000_000, "plx_decode_kernel<128,2,3,2,0>, capture at B=16 (887.0 MB for 883.04 MB of K/V) scaled by the key count"),
+    "C6": (2 * 541_600_000, "plx_decode_kernel<64,2,2,4,0>, capture at B=32 scaled x2 (before the prologue change)"),
+    "P1": (8 * 51_000_000, "plx_prefill_kernel<true,128>, capture at B=1 scaled x8"),
     "T1": (4 * 513_000_000, "plx_bwd_prep/row/col kernels, capture at B=2 scaled x4"),
 }
 NCU_TRAFFIC_FP8 = {"C3": (2 * 540_800_000, "plx_decode_kernel<128,2,2,4,fp8>, capture at B=32 scaled x2")}
