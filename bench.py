@@ -453,7 +453,7 @@ def run_ours(args, rank, world, local_rank):
                     "around the device call: this variant has no host-buffer entry point); "
                     if (args.page_size or args.fp8_kv or Lq > 1) else
                     "q and r read from pinned host memory and the output written to pinned host memory every step "
-                    "(by the library's staging kernel and by the attention kernel itself, over the host link); ") +
+                    "(both by the attention kernel itself, over the host link: one launch, no copy command); ") +
                    "the KV cache is device-resident state of a decode step", **timing_note(t_e2e)}
     clocks = t_call["clocks"]
 

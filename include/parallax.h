@@ -224,11 +224,12 @@ int parallax_decode_combine_gathered(const float* partials, void* out, int B, in
  * out_host, and SYNCHRONISES `stream` before returning.  The KV cache and seqlens
  * stay device pointers: the cache is resident state of a decode step, not a
  * per-step input.  Page-locked (device-mapped) host memory takes a shorter route:
- * q_host and r_host are read over the host link by one staging kernel (16-byte
- * aligned buffers) on which the attention kernel is launched as a programmatic
- * dependent, and the attention kernel writes out_host itself, so the step has
- * no copy command at all; pageable memory is staged with copy commands.  The
- * result is the same bits either way.
+ * the attention kernel reads q_host and r_host itself (16-byte aligned buffers:
+ * every CTA fetches its own rows over the host link into shared memory, so the
+ * transfer of later CTAs' rows overlaps the streaming of the earlier ones) and
+ * writes out_host itself, so the step is ONE launch with no copy command at all;
+ * pageable memory is staged with copy commands.  The result is the same bits
+ * either way.
  */
 int parallax_decode_fwd_host(const void* q_host, const void* r_host, const void* k_cache,
                              const void* v_cache, const int32_t* seqlens, void* out_host, int B,

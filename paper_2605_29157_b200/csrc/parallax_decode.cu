@@ -118,6 +118,10 @@ struct KernelParams {
     // let the next kernel of the stream start early from this kernel's first instruction on (grids that fill
     // every CTA slot of the device) instead of from its last
     int signal_early = 0;
+    // q and r live in page-locked host memory (host-buffer entry): every CTA fetches its group's rows once with
+    // 16-byte loads into shared memory (coalesced requests over the host link) instead of building its fragments
+    // from 4-byte global loads
+    int qr_staged = 0;
     // What the host knows about the buffers, for the index checks of the debug build (PLX_DEBUG_CHECKS):
     // rows each K/V tensor map covers, and the number of records `partials` has room for.
     long long kv_rows = 0;
@@ -377,8 +381,9 @@ struct SmemLayout {
     static constexpr int kTensorBytes = kHalves * kHalfBytes; // K (or V) tile
     static constexpr int kStageBytes = 2 * kTensorBytes;      // K tile then V tile
     static constexpr int kRingBytes = kWarps * NSTAGES * kStageBytes;
-    static constexpr int kBarrierBytes = (kWarps * NSTAGES + 1) * 8;  // + one for the split-merge staging
-    static constexpr int kTotalBytes = 1024 + kRingBytes + kBarrierBytes + PLX_SMEM_PAD;  // 1024: alignment slack
+    static constexpr int kBarrierBytes = ((kWarps * NSTAGES + 1) * 8 + 15) / 16 * 16;  // + one for the split-merge staging
+    static constexpr int kQrBytes = 2 * 8 * D * 2;  // q and r rows of up to eight heads (host-resident q, r are staged here)
+    static constexpr int kTotalBytes = 1024 + kRingBytes + kBarrierBytes + kQrBytes + PLX_SMEM_PAD;  // 1024: alignment slack
 };
 
 // FP8: the caches hold e4m3 bytes ([rows, D] bytes, D = 128); tiles are converted exactly to fp16 in
@@ -571,12 +576,23 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     // second head pair of a quad takes the four columns a single pair leaves empty, so one MMA per k-step
     // scores four heads.
     uint32_t bqr[NQ][KSTEPS][2];
+    const __nv_bfloat16* q_rows = p.q + (static_cast<size_t>(b) * p.Hq + hkv * G) * D;  // the group's G rows are contiguous
+    const __nv_bfloat16* r_rows = p.r + (static_cast<size_t>(b) * p.Hq + hkv * G) * D;
+    if (p.qr_staged) {  // CTA-uniform
+        constexpr int kN16 = G * D * 2 / 16;  // 16-byte words per tensor
+        uint4* const sq = reinterpret_cast<uint4*>(smem + SL::kRingBytes + SL::kBarrierBytes);
+        for (int i = threadIdx.x; i < 2 * kN16; i += kThreads)
+            sq[i] = i < kN16 ? reinterpret_cast<const uint4*>(q_rows)[i] : reinterpret_cast<const uint4*>(r_rows)[i - kN16];
+        __syncthreads();
+        q_rows = reinterpret_cast<const __nv_bfloat16*>(sq);
+        r_rows = reinterpret_cast<const __nv_bfloat16*>(sq + kN16);
+    }
 #pragma unroll
     for (int qd = 0; qd < NQ; ++qd) {
         const int n = lane >> 2;
         const int hl = 4 * qd + 2 * (n >> 2) + (n & 1);
         const __nv_bfloat16* src = nullptr;
-        if (hl < G) src = ((n & 2) ? p.r : p.q) + (static_cast<size_t>(b) * p.Hq + hkv * G + hl) * D;
+        if (hl < G) src = ((n & 2) ? r_rows : q_rows) + hl * D;
 #pragma unroll
         for (int ks = 0; ks < KSTEPS; ++ks) {
             if constexpr (FP8) {
@@ -1445,23 +1461,6 @@ int plx_combine_after_producer(const float* partials, void* out, int rows, int D
     return launch_combine(partials, nullptr, nullptr, 0, 0, out, 1, rows, D, num_splits, out_dtype, stream, 1, true);
 }
 
-// Host-buffer entry point: q and r read straight out of page-locked, device-mapped host memory with
-// 16-byte loads into the workspace (one launch instead of two copy commands, each with its own fixed
-// latency).  The attention kernel is launched as a programmatic dependent of this one.
-__global__ void __launch_bounds__(256) plx_stage_inputs_kernel(const uint4* __restrict__ q_host,
-                                                                const uint4* __restrict__ r_host,
-                                                                uint4* __restrict__ q_dev, uint4* __restrict__ r_dev,
-                                                                size_t n16)
-{
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (i < n16) {
-        const uint4 a = q_host[i], b = r_host[i];
-        q_dev[i] = a;
-        r_dev[i] = b;
-    }
-}
-
 // device view of page-locked, device-mapped host memory (nullptr for pageable memory or device pointers)
 static void* mapped_host_view(const void* host)
 {
@@ -1556,7 +1555,8 @@ static int decode_fwd_impl(const void* q, const void* r, const void* k_cache, co
                            float scale, int out_dtype, void* workspace, size_t workspace_bytes, int num_splits,
                            void* stream, const int32_t* block_table, int page_size, int max_pages, uint64_t kv_rows,
                            bool fp8 = false, float k_scale = 1.0f, float v_scale = 1.0f, bool dependent_launch = false,
-                           const float* k_scales = nullptr, const float* v_scales = nullptr, int lq = 1)
+                           const float* k_scales = nullptr, const float* v_scales = nullptr, int lq = 1,
+                           bool qr_staged = false)
 {
     int rc = check_inputs(q, r, k_cache, v_cache, B, Hq, Hkv, D, T_max);
     if (rc != PLX_OK) return rc;
@@ -1614,6 +1614,7 @@ static int decode_fwd_impl(const void* q, const void* r, const void* k_cache, co
     }
     kp.dependent_launch = dependent_launch ? 1 : 0;
     kp.lq = lq;
+    kp.qr_staged = qr_staged ? 1 : 0;
     const int max_g = fp8 ? 4 : 8;  // the e4m3 variant is built for up to four heads per CTA
     kp.kv_rows = static_cast<long long>(rows);
     if (partials)
@@ -1959,21 +1960,18 @@ int parallax_decode_fwd_host(const void* q_host, const void* r_host, const void*
         if (ns_eff > 1 && workspace_bytes < fixed_bytes(B, Hq, D) + partial_bytes(B, Hq, D, ns_eff)) return PLX_ERR_WORKSPACE;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (in_direct) {
-        const size_t n16 = n * 2 / 16;
-        plx_stage_inputs_kernel<<<static_cast<unsigned>((n16 + 255) / 256), 256, 0, st>>>(
-            static_cast<const uint4*>(q_view), static_cast<const uint4*>(r_view), static_cast<uint4*>(q_dev),
-            static_cast<uint4*>(r_dev), n16);
-        if (cudaGetLastError() != cudaSuccess) return PLX_ERR_CUDA;
-    } else {
+    // Page-locked, device-mapped q and r are not copied at all: the attention kernel's CTAs fetch their own rows over
+    // the host link (16-byte loads into shared memory, once per CTA), so the transfer of a later CTA's rows
+    // overlaps the K/V streaming of the earlier ones instead of standing in front of the whole kernel.
+    if (!in_direct) {
         if (cudaMemcpyAsync(q_dev, q_host, n * 2, cudaMemcpyHostToDevice, st) != cudaSuccess) return PLX_ERR_CUDA;
         if (cudaMemcpyAsync(r_dev, r_host, n * 2, cudaMemcpyHostToDevice, st) != cudaSuccess) return PLX_ERR_CUDA;
     }
     rc = big_group ? parallax_decode_fwd_ex(q_dev, r_dev, k_cache, v_cache, seqlens, out_dev, B, Hq, Hkv, D, T_max, scale,
                                             out_dtype, workspace, workspace_bytes, num_splits, stream)
-                   : decode_fwd_impl(q_dev, r_dev, k_cache, v_cache, seqlens, out_dev, B, Hq, Hkv, D, T_max, scale,
-                                     out_dtype, workspace, workspace_bytes, num_splits, stream, nullptr, 0, 0, 0, false,
-                                     1.0f, 1.0f, in_direct);
+                   : decode_fwd_impl(in_direct ? q_view : q_dev, in_direct ? r_view : r_dev, k_cache, v_cache, seqlens, out_dev,
+                                     B, Hq, Hkv, D, T_max, scale, out_dtype, workspace, workspace_bytes, num_splits, stream,
+                                     nullptr, 0, 0, 0, false, 1.0f, 1.0f, false, nullptr, nullptr, 1, in_direct);
     if (rc != PLX_OK) return rc;
     const size_t out_bytes = n * (out_dtype == PLX_OUT_F32 ? 4 : 2);
     if (!out_direct &&
