@@ -145,12 +145,31 @@ __device__ __forceinline__ unsigned long long plx_now()
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
+#define PLX_PHASE_DECL long long ph_t = clock64(), ph_acc[4] = {0, 0, 0, 0}
+#define PLX_PHASE(i)                     \
+    do {                                 \
+        const long long now = clock64(); \
+        ph_acc[i] += now - ph_t;         \
+        ph_t = now;                      \
+    } while (0)
+#define PLX_PHASE_STORE                                                                                   \
+    do {                                                                                                  \
+        if (threadIdx.x == 0 && blockIdx.x < 8)                                                           \
+            for (int i = 0; i < 4; ++i) g_plx_trace[8192 * 5 - 64 + blockIdx.x * 4 + i] = ph_acc[i];      \
+    } while (0)
 #define PLX_STAMP(slot)                                                                  \
     do {                                                                                 \
         if (threadIdx.x == 0 && blockIdx.x < 8192) g_plx_trace[blockIdx.x * 5 + (slot)] = plx_now(); \
     } while (0)
 #else
 #define PLX_STAMP(slot) \
+    do {                \
+    } while (0)
+#define PLX_PHASE_DECL
+#define PLX_PHASE(i) \
+    do {             \
+    } while (0)
+#define PLX_PHASE_STORE \
     do {                \
     } while (0)
 #endif
@@ -642,12 +661,14 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     bool failed = false;
     int s = 0;
     uint32_t parity = 0;
+    PLX_PHASE_DECL;
     for (int n = 0; n < n_my; ++n) {
         const uint32_t bar = bars + 8 * s;
         if (!mbar_wait_bounded(bar, parity)) {
             failed = true;
             break;
         }
+        PLX_PHASE(0);
         if (n == 0) PLX_STAMP(1);
         const uint32_t sK = ring + s * SL::kStageBytes;
         const uint32_t sV = sK + SL::kTensorBytes;
@@ -706,6 +727,7 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 #pragma unroll
             for (int j = 0; j < 4; ++j) c[qd][j] += c2[qd][j];
 
+        PLX_PHASE(1);
         // ---- online softmax state and P^T fragments -----------------------------------------
         uint32_t pb0[NQ], pb1[NQ];   // P^T fragments (bf16 / fp16 parts; with up to two heads also the residuals)
         uint32_t pr0[NQ], pr1[NQ];   // more than two heads: the rounding residuals, a second MMA into the same accumulator
@@ -839,6 +861,7 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             }
         }
 
+        PLX_PHASE(2);
         // ---- O^T += V_c^T . P^T -------------------------------------------------------------
         if constexpr (FP8) {
 #pragma unroll
@@ -898,9 +921,11 @@ plx_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             s = 0;
             parity ^= 1u;
         }
+        PLX_PHASE(3);
     }
 
     PLX_STAMP(2);
+    PLX_PHASE_STORE;
     if (failed) {
         // A wait ran out: record it, give the copies still in flight one more bounded chance to
         // land before this CTA's shared memory is released, and fall through with what we have.
