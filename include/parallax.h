@@ -271,7 +271,7 @@ int parallax_prefill_fwd(const void* q, const void* r, const void* k_cache, cons
  * exactly to fp16, the products run as fp16 x fp16 -> fp32 MMAs (q and r are converted bf16 -> fp16:
  * exact for magnitudes in [6.1e-5, 65504]), the weights reach the value product as fp16 plus fp16
  * residual.  D in {64, 128} (at D = 64 the rows are 64 bytes: the compute-matched shape of Sec. 3.3
- * "Profiling Result"); groups above four heads per KV head are served by several CTAs of at most four.
+ * "Profiling Result"); up to eight heads per KV head are served by one CTA, as with a 16-bit cache.
  * PLX_ERR_BAD_SHAPE if a scale is not a
  * positive finite number.
  */

@@ -1364,11 +1364,19 @@ int dispatch_main(int D, int G, const CUtensorMap& tmK, const CUtensorMap& tmV, 
             if (G == 2) return launch_main<128, 2, PLX_STAGES_FP8, kCtasPerSmFp8, true>(tmK, tmV, kp, stream);
             if (G == 3) return launch_main<128, 3, PLX_STAGES_FP8, 2, true>(tmK, tmV, kp, stream);
             if (G == 4) return launch_main<128, 4, PLX_STAGES_FP8, 2, true>(tmK, tmV, kp, stream);
+            if (G == 5) return launch_main<128, 5, PLX_STAGES_FP8, 2, true>(tmK, tmV, kp, stream);
+            if (G == 6) return launch_main<128, 6, PLX_STAGES_FP8, 2, true>(tmK, tmV, kp, stream);
+            if (G == 7) return launch_main<128, 7, PLX_STAGES_FP8, 2, true>(tmK, tmV, kp, stream);
+            if (G == 8) return launch_main<128, 8, PLX_STAGES_FP8, 2, true>(tmK, tmV, kp, stream);
         } else if (D == 64) {
             if (G == 1) return launch_main<64, 1, PLX_STAGES_FP8, kCtasPerSmFp8, true>(tmK, tmV, kp, stream);
             if (G == 2) return launch_main<64, 2, PLX_STAGES_FP8, kCtasPerSmFp8, true>(tmK, tmV, kp, stream);
             if (G == 3) return launch_main<64, 3, PLX_STAGES_FP8, kCtasPerSmFp8, true>(tmK, tmV, kp, stream);
             if (G == 4) return launch_main<64, 4, PLX_STAGES_FP8, kCtasPerSmFp8, true>(tmK, tmV, kp, stream);
+            if (G == 5) return launch_main<64, 5, PLX_STAGES_FP8, 3, true>(tmK, tmV, kp, stream);
+            if (G == 6) return launch_main<64, 6, PLX_STAGES_FP8, 3, true>(tmK, tmV, kp, stream);
+            if (G == 7) return launch_main<64, 7, PLX_STAGES_FP8, 3, true>(tmK, tmV, kp, stream);
+            if (G == 8) return launch_main<64, 8, PLX_STAGES_FP8, 3, true>(tmK, tmV, kp, stream);
         }
         return PLX_ERR_UNSUPPORTED;
     }
@@ -1594,7 +1602,7 @@ static int decode_fwd_impl(const void* q, const void* r, const void* k_cache, co
     if (num_splits == 0) {
         int sms = 0;
         if ((rc = device_sm_count(&sms)) != PLX_OK) return rc;
-        plan_splits(B, virtual_kv_heads(Hq, Hkv, fp8 ? 4 : 8), D, T_max, sms, seqlens != nullptr, &chunk_len, &ns, fp8);
+        plan_splits(B, virtual_kv_heads(Hq, Hkv), D, T_max, sms, seqlens != nullptr, &chunk_len, &ns, fp8);
         // never plan beyond what the caller's workspace can hold
         if (ns > 1) {
             const size_t fixed = fixed_bytes(B, Hq, D);
@@ -1640,7 +1648,7 @@ static int decode_fwd_impl(const void* q, const void* r, const void* k_cache, co
     kp.dependent_launch = dependent_launch ? 1 : 0;
     kp.lq = lq;
     kp.qr_staged = qr_staged ? 1 : 0;
-    const int max_g = fp8 ? 4 : 8;  // the e4m3 variant is built for up to four heads per CTA
+    const int max_g = 8;
     kp.kv_rows = static_cast<long long>(rows);
     if (partials)
         kp.partial_records = static_cast<long long>((workspace_bytes - fixed_bytes(B, Hq, D)) / ((2 * D + 4) * sizeof(float)));

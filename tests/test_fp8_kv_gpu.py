@@ -40,7 +40,7 @@ def run_case(plx, oracle, cfg, out_dtype=torch.float32, num_splits=0, poison=Fal
 
 
 @pytest.mark.parametrize("D", [128, 64])
-@pytest.mark.parametrize("G", [1, 2, 3, 4])
+@pytest.mark.parametrize("G", [1, 2, 3, 4, 5, 6, 7, 8])
 @pytest.mark.parametrize("T", [1, 2, 15, 16, 17, 63, 64, 65, 127, 300, 1000])
 def test_fp8_shape_sweep_single_split(plx, oracle, D, G, T):
     """D = 64: 64-byte cache rows, staged in boxes with the 64-byte swizzle."""
@@ -48,7 +48,7 @@ def test_fp8_shape_sweep_single_split(plx, oracle, D, G, T):
     run_case(plx, oracle, cfg, num_splits=1)
 
 
-@pytest.mark.parametrize("D,G", [(128, 1), (128, 2), (128, 4), (64, 2), (64, 3)])
+@pytest.mark.parametrize("D,G", [(128, 1), (128, 2), (128, 4), (64, 2), (64, 3), (128, 7), (64, 8)])
 @pytest.mark.parametrize("T,ns", [(130, 2), (1000, 3), (4096, 0), (5000, 7), (12800, 120)])
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
 def test_fp8_split_kv(plx, oracle, D, G, T, ns, out_dtype):
@@ -58,7 +58,7 @@ def test_fp8_split_kv(plx, oracle, D, G, T, ns, out_dtype):
 
 def test_fp8_head_dim_64_ragged_paged_and_groups_above_four(plx, oracle):
     """The compute-matched shape over an e4m3 cache: ragged lengths with NaN padding, a paged cache, and a
-    group of eight query heads (two CTAs of four per KV head in this variant)."""
+    group of eight query heads (one CTA per KV head, two accumulator sets)."""
     cfg = wl.DecodeConfig("fp8 d64 ragged", B=5, Hq=16, Hkv=2, D=64, T_max=2500, ragged=(1, 2500), seed=955)
     run_case(plx, oracle, cfg, poison=True)
     x = wl.make_inputs(cfg, "cuda", poison_padding=True)
