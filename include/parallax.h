@@ -34,11 +34,20 @@
  *     seqlens[b] == 0 gives a row of zeros.  The new token's own key and value are
  *     expected to be in the cache already and counted by seqlens.
  *   - Supported shapes: D in {64, 128}; Hq a multiple of Hkv with group size
- *     Hq/Hkv from 1 to 64 (groups of 5 to 8 are served by several CTAs per KV head, at most
- *     four query heads each; parallax_decode_fwd_ex and parallax_decode_fwd_paged hand groups
- *     above 8 -- multi-query models -- to the tensor-core kernel, see
- *     parallax_decode_fwd_multi, which also lifts the limit of 64); q, r, out 4-byte
+ *     Hq/Hkv from 1 to 64 (up to eight query heads of a KV head are served by one CTA;
+ *     larger groups by several CTAs per KV head, or -- parallax_decode_fwd_ex and
+ *     parallax_decode_fwd_paged route them by measured crossover -- by the tensor-core kernel,
+ *     see parallax_decode_fwd_multi, which also lifts the limit of 64); q, r, out 4-byte
  *     aligned; k_cache, v_cache 16-byte aligned; workspace 16-byte aligned.
+ *   - Launch ordering: the decode kernels are launched with the programmatic stream
+ *     serialisation attribute (they wait, before they touch memory, for the kernel
+ *     before them in the stream) and signal their own dependents early, so that
+ *     back-to-back decode calls overlap a call's launch with its predecessor's tail.
+ *     For a kernel launched the ordinary way after a call nothing changes: it starts
+ *     when the call's kernels have completed.  A kernel that the CALLER launches as
+ *     a programmatic dependent after a decode call may be scheduled before that
+ *     call has completed and has to execute cudaGridDependencySynchronize() before
+ *     it touches the call's output, as that launch mode requires of any kernel.
  *   - Thread safety: entry points may be called from several host threads;
  *     parallax_set_layout / parallax_decode_fwd share one process-wide default.
  */
