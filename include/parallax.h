@@ -262,7 +262,9 @@ int parallax_workspace_status(const void* workspace, int32_t* status_host, void*
  * Supported: D in {64, 128}, any Hq multiple of Hkv; all tensors 16-byte aligned.
  * p_precision: PLX_P_BF16_RESIDUAL keeps the decode path's accuracy (the weights reach the value
  * product as bf16 plus residual, at the price of two extra MMAs per tile); PLX_P_BF16 sends plain
- * bf16 weights, the precision of a conventional bf16 attention kernel.
+ * bf16 weights, the precision of a conventional bf16 attention kernel; PLX_P_BF16_ADAPTIVE keeps the
+ * residual products only in the row tiles in which some row sees fewer than PLX_P_ADAPTIVE_MIN_KEYS keys
+ * (two launches: the plain build and the residual build, each over its own tiles).
  * `status` is an optional device int32 set non-zero if a bounded device-side wait
  * ran out (NULL = not recorded).  One launch, no workspace.
  */
