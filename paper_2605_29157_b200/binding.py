@@ -124,13 +124,22 @@ def _check(rc: int) -> None:
 
 
 def _ptr(t: Optional[torch.Tensor]):
-    return None if t is None else ctypes.c_void_p(t.data_ptr())
+    # a plain int: the argument types are declared, so ctypes converts it without an intermediate object
+    return None if t is None else t.data_ptr()
 
 
-def _stream(stream) -> ctypes.c_void_p:
+_raw_current_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+
+
+def _stream(stream):
+    """cudaStream_t as an int (0 = the legacy default stream).  Without an argument: torch's current stream of the
+    current device, through torch's raw-handle accessor where it exists (building a Stream object costs about 4 us,
+    which a launch-bound decode call notices)."""
     if stream is None:
+        if _raw_current_stream is not None:
+            return _raw_current_stream(torch.cuda.current_device()) or None
         stream = torch.cuda.current_stream()
-    return ctypes.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+    return (stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)) or None
 
 
 def _out_dtype_code(dtype: torch.dtype) -> int:
@@ -421,7 +430,7 @@ def parallax_decode_fwd_args(q, r, k_cache, v_cache, seqlens, out, scale, block_
     if workspace is not None:
         a.workspace, a.workspace_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
     a.num_splits = int(num_splits)
-    a.stream = _stream(stream).value
+    a.stream = _stream(stream)
     _check(_lib.parallax_decode_fwd_args(ctypes.byref(a)))
     return out
 
