@@ -537,3 +537,20 @@ def test_multi_query_groups_go_to_the_tensor_core_kernel(plx, oracle, D, Hq, Hkv
     oh = torch.full((cfg.B, cfg.Hq, cfg.D), float("nan"), dtype=torch.float32).pin_memory()
     plx.parallax_decode_fwd_host(qh, rh, x["k"], x["v"], x["seqlens"], oh, cfg.scale, ws, ns)
     assert_parity(oh.numpy(), want, torch.float32, "host entry")
+
+
+def test_one_million_key_context(plx, oracle):
+    """One sequence of 2^20 keys (4 GiB of K and V): split planning, chunk arithmetic and the fused merge at a
+    context eight times the longest benchmark configuration; sampled rows against the oracle, every row finite."""
+    cfg = wl.DecodeConfig("1M", B=1, Hq=16, Hkv=8, D=128, T_max=1 << 20, seed=4321)
+    x = wl.make_inputs(cfg, "cuda")
+    out = torch.full((cfg.B, cfg.Hq, cfg.D), float("nan"), dtype=torch.float32, device="cuda")
+    ws = plx.alloc_workspace(cfg.B, cfg.Hq, cfg.D, plx.PLX_MAX_SPLITS, "cuda")
+    plx.parallax_decode_fwd_ex(x["q"], x["r"], x["k"], x["v"], None, out, cfg.scale, ws, 0)
+    torch.cuda.synchronize()
+    assert plx.parallax_workspace_status(ws) == 0
+    assert torch.isfinite(out).all()
+    rows = [(0, 0), (0, 7), (0, 15)]
+    want = oracle_rows(oracle, x, cfg.scale, rows)
+    got = np.stack([out[b, h].cpu().numpy() for (b, h) in rows])
+    assert_parity(got, want, torch.float32, "2^20 keys")
