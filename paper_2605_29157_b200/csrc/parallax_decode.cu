@@ -1231,6 +1231,12 @@ int virtual_kv_heads(int Hq, int Hkv, int max_g = 8)
     split_group(Hq / Hkv, &g, &kv_div, max_g);
     return Hkv * kv_div;
 }
+int heads_per_cta(int Hq, int Hkv)
+{
+    int g = 1, kv_div = 1;
+    split_group(Hq / Hkv, &g, &kv_div);
+    return g;
+}
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
 // Split plan.  Cost model in units of "time for one resident CTA to stream one key while the device
@@ -1249,15 +1255,22 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) &
 // key there (100), and a split plan pays ~220 + 6 per split for the merge and the second generation.
 // The e4m3 kernel spends twice the instructions per byte, so it needs nearly all four CTAs of an SM to
 // saturate HBM (cap 1.5: 384 resident CTAs reach 6.0 TB/s where 512 reach 6.6) and its fixed cost is 140.
-double plan_cost(int chunk, int ns_eff, long long streams, long long slots, bool ragged, int D, bool fp8 = false)
+// Five to eight heads per CTA (D = 128, 16-bit cache) have constants of their own: a tile costs such a warp ~1560
+// cycles instead of ~1170, so a CTA alone on its SM pulls less and the partial-wave speed-up is capped at 1.4; fixed cost
+// 200 per CTA generation, merge 150 + 10 per split.  Fitted on a sweep of 14 (batch, context) cells x the split counts
+// that give 74...592 CTAs: the plan then loses 0.2-1 % on average against the best measured split count, where the
+// two-head constants lost 11 % (worst cell 30 %: 16 x 8192 keys was not split, 118 against 93 us).
+double plan_cost(int chunk, int ns_eff, long long streams, long long slots, bool ragged, int D, bool fp8 = false,
+                 int heads_per_cta = 2)
 {
     const long long ctas = streams * ns_eff;
     const long long full = ctas / slots, last = ctas % slots;
     const bool small_stage = D < 128 || fp8;  // 4 KiB stages, four CTAs per SM
-    const double fixed = fp8 ? 140.0 : small_stage ? 100.0 : 60.0;
+    const bool many_heads = !small_stage && heads_per_cta >= 5;
+    const double fixed = fp8 ? 140.0 : small_stage ? 100.0 : many_heads ? 200.0 : 60.0;
     double cost = static_cast<double>(full) * chunk + fixed * static_cast<double>(ctas) / static_cast<double>(slots) + fixed;
     if (last > 0) {
-        const double cap = fp8 ? 1.5 : small_stage ? 1.9 : 2.2;
+        const double cap = fp8 ? 1.5 : small_stage ? 1.9 : many_heads ? 1.4 : 2.2;
         const double speedup = static_cast<double>(slots) / static_cast<double>(last);
         double tail = chunk / (speedup < cap ? speedup : cap);
         if (small_stage) {
@@ -1268,13 +1281,13 @@ double plan_cost(int chunk, int ns_eff, long long streams, long long slots, bool
         }
         cost += tail;
     }
-    if (ns_eff > 1) cost += small_stage ? 220.0 + 6.0 * ns_eff : 300.0 + 2.3 * ns_eff;
+    if (ns_eff > 1) cost += small_stage ? 220.0 + 6.0 * ns_eff : many_heads ? 150.0 + 10.0 * ns_eff : 300.0 + 2.3 * ns_eff;
     if (ragged) cost += chunk;
     return cost;
 }
 
 void plan_splits(int B, int Hkv, int D, int T_max, int num_sms, bool ragged, int* chunk_len, int* num_splits,
-                 bool fp8 = false)
+                 bool fp8 = false, int heads_per_cta = 2)
 {
     const long long streams = static_cast<long long>(B) * Hkv;
     const long long slots = static_cast<long long>(num_sms) * (fp8 ? kCtasPerSmFp8 : D == 64 ? PLX_CTAS_PER_SM_D64 : kCtasPerSm);
@@ -1290,7 +1303,7 @@ void plan_splits(int B, int Hkv, int D, int T_max, int num_sms, bool ragged, int
         prev_chunk = chunk;
         if (ns > 1 && chunk < kMinChunk) break;
         const int ns_eff = (T_max + chunk - 1) / chunk;
-        const double cost = plan_cost(chunk, ns_eff, streams, slots, ragged, D, fp8);
+        const double cost = plan_cost(chunk, ns_eff, streams, slots, ragged, D, fp8, heads_per_cta);
         if (best_cost < 0.0 || cost < best_cost * 0.995) {  // ties go to fewer splits
             best_cost = cost;
             best_chunk = chunk;
@@ -1540,7 +1553,8 @@ int parallax_decode_plan(int B, int Hq, int Hkv, int D, int T_max, int num_sms, 
 {
     if (!chunk_len || !num_splits) return PLX_ERR_NULL_POINTER;
     if (!shape_ok(B, Hq, Hkv, D) || T_max <= 0 || num_sms <= 0) return PLX_ERR_BAD_SHAPE;
-    plan_splits(B, virtual_kv_heads(Hq, Hkv), D, T_max, num_sms, has_seqlens != 0, chunk_len, num_splits);
+    plan_splits(B, virtual_kv_heads(Hq, Hkv), D, T_max, num_sms, has_seqlens != 0, chunk_len, num_splits, false,
+                heads_per_cta(Hq, Hkv));
     return PLX_OK;
 }
 
@@ -1602,7 +1616,7 @@ static int decode_fwd_impl(const void* q, const void* r, const void* k_cache, co
     if (num_splits == 0) {
         int sms = 0;
         if ((rc = device_sm_count(&sms)) != PLX_OK) return rc;
-        plan_splits(B, virtual_kv_heads(Hq, Hkv), D, T_max, sms, seqlens != nullptr, &chunk_len, &ns, fp8);
+        plan_splits(B, virtual_kv_heads(Hq, Hkv), D, T_max, sms, seqlens != nullptr, &chunk_len, &ns, fp8, heads_per_cta(Hq, Hkv));
         // never plan beyond what the caller's workspace can hold
         if (ns > 1) {
             const size_t fixed = fixed_bytes(B, Hq, D);
@@ -2087,7 +2101,7 @@ extern "C" int parallax_decode_fwd_static(const void* q, const void* r, const vo
     if (num_splits == 0) {
         int sms = 0;
         if ((rc = device_sm_count(&sms)) != PLX_OK) return rc;
-        plan_splits(B, virtual_kv_heads(Hq, Hkv), D, T_max, sms, seqlens != nullptr, &chunk_len, &ns);
+        plan_splits(B, virtual_kv_heads(Hq, Hkv), D, T_max, sms, seqlens != nullptr, &chunk_len, &ns, false, heads_per_cta(Hq, Hkv));
         // the planner may only use as many splits as the fixed array can hold
         while (ns > 1 && partial_bytes(B, Hq, D, ns) > PLX_STATIC_SCRATCH_BYTES) {
             --ns;
