@@ -1260,6 +1260,14 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) &
 // 200 per CTA generation, merge 150 + 10 per split.  Fitted on a sweep of 14 (batch, context) cells x the split counts
 // that give 74...592 CTAs: the plan then loses 0.2-1 % on average against the best measured split count, where the
 // two-head constants lost 11 % (worst cell 30 %: 16 x 8192 keys was not split, 118 against 93 us).
+// CTAs of a build that fit on one SM (registers and shared memory; mirrors the launch bounds in dispatch_main)
+int resident_ctas(int D, bool fp8, int heads_per_cta)
+{
+    if (fp8) return D == 128 ? (heads_per_cta <= 2 ? kCtasPerSmFp8 : 2) : (heads_per_cta <= 4 ? kCtasPerSmFp8 : 3);
+    if (D == 64) return heads_per_cta <= 4 ? PLX_CTAS_PER_SM_D64 : 3;
+    return kCtasPerSm;
+}
+
 double plan_cost(int chunk, int ns_eff, long long streams, long long slots, bool ragged, int D, bool fp8 = false,
                  int heads_per_cta = 2)
 {
@@ -1267,21 +1275,28 @@ double plan_cost(int chunk, int ns_eff, long long streams, long long slots, bool
     const long long full = ctas / slots, last = ctas % slots;
     const bool small_stage = D < 128 || fp8;  // 4 KiB stages, four CTAs per SM
     const bool many_heads = !small_stage && heads_per_cta >= 5;
-    const double fixed = fp8 ? 140.0 : small_stage ? 100.0 : many_heads ? 200.0 : 60.0;
+    // D = 64, 16-bit cache, five to eight heads per CTA (three CTAs per SM): cap 1.2, fixed cost 300, 10 per split,
+    // uneven-spread factor 0.6 (same sweep at D = 64: plan loss 8 % -> 0.1 % on the measured split counts)
+    const bool many_heads_d64 = !fp8 && D < 128 && heads_per_cta >= 5;
+    const double fixed = fp8 ? 140.0 : many_heads_d64 ? 300.0 : small_stage ? 100.0 : many_heads ? 200.0 : 60.0;
     double cost = static_cast<double>(full) * chunk + fixed * static_cast<double>(ctas) / static_cast<double>(slots) + fixed;
     if (last > 0) {
-        const double cap = fp8 ? 1.5 : small_stage ? 1.9 : many_heads ? 1.4 : 2.2;
+        const double cap = fp8 ? 1.5 : many_heads_d64 ? 1.2 : small_stage ? 1.9 : many_heads ? 1.4 : 2.2;
         const double speedup = static_cast<double>(slots) / static_cast<double>(last);
         double tail = chunk / (speedup < cap ? speedup : cap);
         if (small_stage) {
             // With four CTAs per SM a partial wave that does not spread evenly over the SMs (304 CTAs on
             // 148 SMs: eight SMs hold three) finishes with its fullest SMs; measured ~14 % for that case.
-            const double per_sm = static_cast<double>(last) * PLX_CTAS_PER_SM_D64 / static_cast<double>(slots);
-            tail *= 1.0 + 0.3 * (ceil(per_sm) / per_sm - 1.0);
+            const double per_sm = static_cast<double>(last) * resident_ctas(D, fp8, heads_per_cta) / static_cast<double>(slots);
+            tail *= 1.0 + (many_heads_d64 ? 0.6 : 0.3) * (ceil(per_sm) / per_sm - 1.0);
         }
         cost += tail;
     }
-    if (ns_eff > 1) cost += small_stage ? 220.0 + 6.0 * ns_eff : many_heads ? 150.0 + 10.0 * ns_eff : 300.0 + 2.3 * ns_eff;
+    if (ns_eff > 1)
+        cost += many_heads_d64 ? 220.0 + 10.0 * ns_eff
+                : small_stage  ? 220.0 + 6.0 * ns_eff
+                : many_heads   ? 150.0 + 10.0 * ns_eff
+                               : 300.0 + 2.3 * ns_eff;
     if (ragged) cost += chunk;
     return cost;
 }
@@ -1290,7 +1305,7 @@ void plan_splits(int B, int Hkv, int D, int T_max, int num_sms, bool ragged, int
                  bool fp8 = false, int heads_per_cta = 2)
 {
     const long long streams = static_cast<long long>(B) * Hkv;
-    const long long slots = static_cast<long long>(num_sms) * (fp8 ? kCtasPerSmFp8 : D == 64 ? PLX_CTAS_PER_SM_D64 : kCtasPerSm);
+    const long long slots = static_cast<long long>(num_sms) * resident_ctas(D, fp8, heads_per_cta);
     const int granules = (T_max + kChunkGranule - 1) / kChunkGranule;
     const int kMinChunk = 256;
     double best_cost = -1.0;
