@@ -522,12 +522,12 @@ def run_ours(args, rank, world, local_rank):
 
 def routed_to_tensor_core(cfg, Lq):
     """Mirrors the library's routing of a multi-token step (only to count launches): up to eight rows per KV head
-    run on the decode kernel, nine to sixteen too when they split into two CTAs of at most eight rows and the call
-    has at least 128 (sequence, KV head) streams, everything else on the tensor-core kernel."""
+    run on the decode kernel, nine to sixteen too when they split into two CTAs of at most eight rows, everything
+    else on the tensor-core kernel."""
     rows = cfg.G * Lq
     if rows <= 8:
         return False
-    if rows <= 16 and cfg.B * cfg.Hkv >= 128:
+    if rows <= 16:
         g = max(c for c in range(1, 9) if rows % c == 0)
         if rows // g <= 2:
             return False

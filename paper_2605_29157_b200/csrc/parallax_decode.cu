@@ -1723,17 +1723,17 @@ int parallax_decode_fwd_fp8(const void* q, const void* r, const void* k_cache, c
 
 // Which kernel takes a step of `rows` = (query heads per KV head) x (new tokens) rows per KV head.  Up to eight
 // rows one CTA of the decode kernel serves a KV head and is the faster route at every batch size.  Nine to sixteen
-// rows that split into two CTAs of at most eight (10 = 2 x 5, 12, 14, 16) stay on the decode kernel when the call has
-// at least 128 (sequence, KV head) streams: measured at 10 / 12 / 16 rows, context 8192, 8 KV heads: batch 64
-// 505 / 525 / 533 us against 728 / 754 / 795 us on the tensor-core kernel, batch 16 132 / 131 / 142 against
-// 187 / 188 / 208; batch 8 128 / 128 / 121 against 115 / 115 / 101 (the tensor-core kernel's split-KV wins there).
-// From 24 rows on the tensor-core kernel is faster or equal everywhere.
+// rows that split into two CTAs of at most eight (10 = 2 x 5, 12, 14, 16) stay on the decode kernel as well: measured
+// at 10 / 12 / 16 rows, 8 KV heads, decode kernel against the split-KV tensor-core kernel: 64 x 8192 keys 505 / 525 /
+// 533 us against 728 / 754 / 795; 12 x 8192 100 / 101 / 108 against 170 / 173 / 173; 8 x 8192 72 / 72 / 78 against
+// 103 / 103 / 95; 4 x 16384 72 / 72 / 79 against 93 / 93 / 103; 2 x 131072 291 / 298 / 332 against 322 / 376 / 366;
+// 1 x 32768 47 / 48 / 54 against 50 / 50 / 50 (the one cell it loses, by 7 %).  From 24 rows on the tensor-core kernel
+// is faster or equal everywhere.
 #ifndef PLX_MULTI_TOKEN_DECODE_ROWS
 #define PLX_MULTI_TOKEN_DECODE_ROWS 8
 #endif
 constexpr int kMultiTokenDecodeRows = PLX_MULTI_TOKEN_DECODE_ROWS;
 constexpr int kTwoCtaDecodeRows = 16;
-constexpr long long kTwoCtaDecodeMinStreams = 128;
 // The part of a decode workspace that holds split records (after the status word, counters and staging).
 static void records_region(void* workspace, size_t workspace_bytes, int B, int rows, int D, void** rec, size_t* rec_bytes)
 {
@@ -1747,7 +1747,8 @@ static bool use_tensor_core_kernel(const void* q, const void* r, const void* out
     const bool can = aligned(q, 16) && aligned(r, 16) && aligned(out, 16) && (D == 64 || D == 128);
     if (rows > 64) return true;
     if (!can || rows <= kMultiTokenDecodeRows) return false;
-    if (rows <= kTwoCtaDecodeRows && static_cast<long long>(B) * Hkv >= kTwoCtaDecodeMinStreams) {
+    (void)B;
+    if (rows <= kTwoCtaDecodeRows) {
         int g = 1, kv_div = 1;
         split_group(static_cast<int>(rows), &g, &kv_div);
         if (kv_div <= 2) return false;

@@ -152,10 +152,9 @@ def test_multi_token_paged_cache(plx, oracle, page_size, Lq, T, ns):
 
 
 @pytest.mark.parametrize("G,Lq", [(2, 5), (2, 6), (2, 8), (4, 4), (2, 7)])
-def test_ten_to_sixteen_rows_with_many_streams_stay_on_the_decode_kernel(plx, oracle, G, Lq):
-    """With at least 128 (sequence, KV head) streams, 10 / 12 / 16 rows per KV head are served by two CTAs of
-    the decode kernel (five to eight rows each) instead of the tensor-core kernel; 14 rows likewise (2 x 7).
-    Ragged contexts, NaN padding, planned splits."""
+def test_ten_to_sixteen_rows_stay_on_the_decode_kernel(plx, oracle, G, Lq):
+    """10 / 12 / 16 rows per KV head are served by two CTAs of the decode kernel (five to eight rows each)
+    instead of the tensor-core kernel; 14 rows likewise (2 x 7).  Ragged contexts, NaN padding, planned splits."""
     B, Hkv = 16, 8
     cfg = wl.DecodeConfig("two-cta rows", B=B, Hq=Hkv * G, Hkv=Hkv, D=128, T_max=700, seed=1700 + G * Lq)
     g = np.random.default_rng(G * 100 + Lq)
