@@ -163,7 +163,7 @@ def test_backward_full_size_in_the_bench_configuration(plx, oracle):
     # RMS bar stays 1e-2, the element bound is taken against the sampled rows' largest entry.
     g = np.random.default_rng(7)
     rows = [(int(g.integers(B)), int(g.integers(Hq)), int(i)) for i in
-            list(g.integers(0, Lq, size=20)) + [0, 1, 63, 64, 127, 128, Lq - 1]]
+            list(g.integers(0, Lq, size=120)) + [0, 1, 63, 64, 127, 128, Lq - 1]]
     got_q, got_r, want_q, want_r = [], [], [], []
     for (b, h, i) in rows:
         hkv = h // G
@@ -223,7 +223,7 @@ def test_backward_full_size_long_sequence(plx, oracle):
 
     g = np.random.default_rng(17)
     rows = [(int(g.integers(B)), int(g.integers(Hq)), int(i)) for i in
-            list(g.integers(0, Lq, size=12)) + [0, 127, 128, Lq - 1]]
+            list(g.integers(0, Lq, size=60)) + [0, 127, 128, Lq - 1]]
     got_q, got_r, want_q, want_r = [], [], [], []
     for (b, h, i) in rows:
         hkv = h // G

@@ -155,7 +155,7 @@ def test_prefill_full_size_in_the_bench_configuration(plx, oracle, name):
     assert torch.isfinite(out.float()).all()
     g = np.random.default_rng(11)
     rows = [(int(g.integers(cfg.B)), int(g.integers(cfg.Hq)), int(i)) for i in
-            list(g.integers(0, Lq, size=40)) + [i for i in (0, 1, 63, 64, 127, 128, Lq - 1) if i < Lq]]
+            list(g.integers(0, Lq, size=300)) + [i for i in (0, 1, 63, 64, 127, 128, Lq - 1) if i < Lq]]
     for (b, h, i) in rows:
         n = cfg.T_max - Lq + i + 1
         hkv = h // cfg.G
