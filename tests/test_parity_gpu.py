@@ -25,7 +25,7 @@ def run_fwd(plx, x, cfg, out_dtype, num_splits=0, dev="cuda"):
 
 
 @pytest.mark.parametrize("D", [64, 128])
-@pytest.mark.parametrize("G", [1, 2, 3, 4])
+@pytest.mark.parametrize("G", [1, 2, 3, 4, 5, 6, 7, 8])
 @pytest.mark.parametrize("T", [1, 2, 15, 16, 17, 63, 64, 65, 127, 300, 1000])
 def test_shape_sweep_single_split(plx, oracle, D, G, T):
     """One CTA per stream, every tail shape of the 16-key tile and the 4-warp round robin."""
@@ -36,7 +36,8 @@ def test_shape_sweep_single_split(plx, oracle, D, G, T):
     assert_parity(got, want, torch.float32, f"D={D} G={G} T={T}")
 
 
-@pytest.mark.parametrize("D,G", [(64, 2), (64, 3), (128, 1), (128, 2), (128, 3), (128, 4)])
+@pytest.mark.parametrize("D,G", [(64, 2), (64, 3), (128, 1), (128, 2), (128, 3), (128, 4), (128, 5), (128, 7), (128, 8),
+                                 (64, 6), (64, 8)])
 @pytest.mark.parametrize("T,ns", [(130, 2), (1000, 3), (1000, 16), (4096, 0), (5000, 7)])
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
 def test_split_kv(plx, oracle, D, G, T, ns, out_dtype):
@@ -48,7 +49,7 @@ def test_split_kv(plx, oracle, D, G, T, ns, out_dtype):
     assert_parity(got, want, out_dtype, f"D={D} G={G} T={T} ns={ns}")
 
 
-@pytest.mark.parametrize("D,G", [(128, 2), (128, 4), (128, 1), (64, 2), (64, 4)])
+@pytest.mark.parametrize("D,G", [(128, 2), (128, 4), (128, 1), (64, 2), (64, 4), (128, 6), (128, 8), (64, 7)])
 def test_many_splits_batched_merge(plx, oracle, D, G):
     """More splits per row than the merging CTA can stage at once (47 records per row at D=128,
     G=2; 23 at G=4): the merge runs in several batches with a running reference exponent.  Ragged
@@ -502,8 +503,8 @@ def test_full_size_every_row_by_a_property(plx, name):
 @pytest.mark.parametrize("D,Hq,Hkv", [(128, 16, 2), (128, 12, 2), (64, 32, 4), (128, 10, 2), (128, 14, 2)])
 @pytest.mark.parametrize("ns", [1, 0, 5])
 def test_large_gqa_groups(plx, oracle, D, Hq, Hkv, ns):
-    """Group sizes above 4 (8, 6, 8, 5, 7 query heads per KV head): a KV head is served by several CTAs of
-    at most four query heads each."""
+    """Group sizes above 4 (8, 6, 8, 5, 7 query heads per KV head): one CTA serves all heads of a KV head
+    (two quads of heads in the 8 MMA columns, each with its own accumulator set)."""
     cfg = wl.DecodeConfig("gqa", B=2, Hq=Hq, Hkv=Hkv, D=D, T_max=1500, ragged=(200, 1500), seed=970 + Hq)
     x = wl.make_inputs(cfg, "cuda", poison_padding=True)
     want = oracle_full(oracle, x, cfg.scale, x["seqlens_host"])
