@@ -291,6 +291,9 @@ def whole_job_value(bytes_per_rank: int, world: int, ms_per_step: float) -> floa
     return bytes_per_rank * world / (ms_per_step * 1e-3) / 1e12
 
 
+PROBE_CALL_BYTES = (128 << 20, 1 << 30)   # the K/V bytes of one C2 call and of one C4 / C6 call
+
+
 def read_probe(dev, stream, sampler):
     """Read-only streaming bandwidth of this GPU, measured in this run with the library's own probe kernel:
     2 GiB buffers, two of them read alternately (4 GiB between two reads of a byte vs 0.123 GiB of L2), each
@@ -317,10 +320,30 @@ def read_probe(dev, stream, sampler):
             call(i)
         t = timer.run(call, 10, min_ms=100.0)
         out[name] = round(nbytes / (t["ms_per_step"] * 1e-3) / 1e9, 1)
+    # The same probe on calls of the size of the smaller decode configurations: a launch that reads 128 MiB
+    # spends a visible part of its time filling and draining the device, so its ceiling is lower than the
+    # 2 GiB figure.  Each call reads the next `size` bytes of the two buffers (4 GiB between two reads of a byte).
+    by_bytes = {}
+    for size in PROBE_CALL_BYTES:
+        per_buf = nbytes // size
+        best_small = 0.0
+        for mode, ctas in ((plx.PLX_PROBE_VECTOR_LOADS, 0), (plx.PLX_PROBE_VECTOR_LOADS, size // 65536),
+                           (plx.PLX_PROBE_BULK_COPIES, 0)):
+            def call(i, mode=mode, ctas=ctas):
+                j = i % (2 * per_buf)
+                src = bufs[j // per_buf][(j % per_buf) * (size // 4):(j % per_buf + 1) * (size // 4)]
+                plx.parallax_read_probe(src, sink, mode, ctas, status, stream)
+            cool_down(0.3)
+            for i in range(3):
+                call(i)
+            t = timer.run(call, 2 * per_buf, min_ms=60.0)
+            best_small = max(best_small, size / (t["ms_per_step"] * 1e-3) / 1e9)
+        by_bytes[str(size)] = round(best_small, 1)
     assert int(status.item()) == 0, "read probe: a bounded wait ran out"
     best = max(out, key=out.get)
     return {"GBps": out, "best": best, "peak": out[best], "bytes_per_launch": nbytes,
-            "l2_policy": "two 2 GiB buffers read alternately"}
+            "l2_policy": "two 2 GiB buffers read alternately",
+            "GBps_by_call_bytes": by_bytes}
 
 
 def describe(cfg, seqlens_host, nsets, chunk, ns):
@@ -509,7 +532,8 @@ def run_ours(args, rank, world, local_rank):
         del sets
         torch.cuda.empty_cache()
         read_peak = roofline.get("peak_read_probe")
-        result["other_configs"] = {n: quick_config(n, sampler, read_peak) for n in sorted(wl.CONFIGS) if n != args.workload}
+        by_bytes = roofline.get("read_probe", {}).get("GBps_by_call_bytes")
+        result["other_configs"] = {n: quick_config(n, sampler, read_peak, by_bytes) for n in sorted(wl.CONFIGS) if n != args.workload}
         result["other_workloads"] = {n: quick_tensor_workload(n, local_rank) for n in ("P2", "T1")}
     if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.fp8_kv and Lq == 1:
         secs, nbytes, threads, desc = oracle_sample_time(cfg, x0, seqlens_host, args.cpu_seconds)
@@ -564,7 +588,7 @@ def graph_replay_us(step, nsets, reps=5):
     return e0.elapsed_time(e1) / (reps * per_graph) * 1e3
 
 
-def quick_config(name, sampler, read_peak=None, steps=20, warmup=5):
+def quick_config(name, sampler, read_peak=None, read_by_bytes=None, steps=20, warmup=5):
     """Device-timed run of one decode configuration (library plan, L2-cold by rotating cache sets, blocks of
     `steps` calls repeated until >= 200 ms of device time): us per call, KV-read TB/s, its fractions of the
     measured copy bandwidth, of this run's read-only probe and of 8 TB/s, and the clocks of its own region."""
@@ -596,6 +620,9 @@ def quick_config(name, sampler, read_peak=None, steps=20, warmup=5):
            "traffic": traffic, "traffic_source": traffic_src, "clocks": t["clocks"], **timing_note(t)}
     if read_peak:
         res["frac_of_read_probe"] = round(kv_bytes / us / 1e3 / read_peak, 4)
+    if read_by_bytes and str(kv_bytes) in read_by_bytes:   # the probe reading exactly this call's bytes per launch
+        res["read_probe_same_bytes_GBps"] = read_by_bytes[str(kv_bytes)]
+        res["frac_of_read_probe_same_bytes"] = round(kv_bytes / us / 1e3 / read_by_bytes[str(kv_bytes)], 4)
     return res
 
 

@@ -31,6 +31,8 @@ def test_decode_line_has_the_contract_keys(cuda_device):
         assert key in r, key
     assert r["bound"] == "hbm" and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-3
     assert 0.2 < r["frac_of_read_probe"] < 1.1                     # a kernel that only reads cannot beat the read probe
+    by_bytes = r["read_probe"]["GBps_by_call_bytes"]               # the probe on calls of C2's and C4's size
+    assert 3000 < by_bytes[str(128 << 20)] < by_bytes[str(1 << 30)] <= 1.02 * r["peak_read_probe"]
     e = d["e2e"]
     assert e["h2d_bytes_per_step"] == 2 * 8 * 16 * 128 * 2 and e["d2h_bytes_per_step"] == 8 * 16 * 128 * 2
     assert 0 < e["value"] <= d["value"] * 1.05                      # end to end is never faster than the device time
