@@ -367,6 +367,22 @@ int parallax_decode_fwd_multi(const void* q, const void* r, const void* k_cache,
                               int T_max, float scale, int out_dtype, void* workspace,
                               size_t workspace_bytes, int num_splits, void* stream);
 
+/*
+ * The same step on the tensor-core kernel that keeps the KEYS on the accumulator lanes (Algorithm 1 with
+ * S^T = K_c [Q; R]^T per 128-key tile and O^T += V_c^T P^T, so the tensor work follows the rows present):
+ * up to 64 rows per KV head (Lq * Hq / Hkv <= 64), D = 128, bf16 caches, contiguous layout; q, r, k_cache,
+ * v_cache, out 16-byte aligned.  Split-KV like parallax_prefill_fwd_ex: `workspace` holds split records only
+ * (parallax_prefill_workspace_bytes(B, Hq, D, Lq, max_splits) bytes, 16-byte aligned; NULL = one split),
+ * num_splits 0 = planned (about one CTA per SM, at least four 128-key tiles per split), records merged by the
+ * decode path's combine kernel on the same stream.  `status` (device int32, may be NULL) receives
+ * PLX_ERR_DEVICE_TIMEOUT if a bounded device-side wait runs out.  PLX_ERR_UNSUPPORTED for other shapes.
+ * parallax_decode_fwd_multi chooses this kernel by itself; this entry forces it.  One or two launches on `stream`.
+ */
+int parallax_decode_fwd_rows(const void* q, const void* r, const void* k_cache, const void* v_cache,
+                             const int32_t* seqlens, void* out, int B, int Hq, int Hkv, int D, int Lq,
+                             int T_max, float scale, int out_dtype, void* workspace, size_t workspace_bytes,
+                             int num_splits, int32_t* status, void* stream);
+
 /* parallax_decode_fwd_multi over the paged cache of parallax_decode_fwd_paged (q, r, out [B, Hq, Lq, D]);
  * the hand-over to the tensor-core kernel needs page_size to be a multiple of 64. */
 int parallax_decode_fwd_multi_paged(const void* q, const void* r, const void* k_pages, const void* v_pages,

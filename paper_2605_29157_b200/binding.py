@@ -53,7 +53,7 @@ EXPORTS = (
     "parallax_decode_step", "parallax_decode_fwd_fp8_per_head", "parallax_decode_fwd_paged_fp8_per_head",
     "parallax_decode_fwd_multi", "parallax_prefill_workspace_bytes", "parallax_prefill_fwd_ex",
     "parallax_prefill_fwd_paged_ex", "parallax_decode_fwd_multi_paged", "parallax_decode_fwd_args",
-    "parallax_read_probe",
+    "parallax_read_probe", "parallax_decode_fwd_rows",
 )
 TEST_HOOK_EXPORTS = ("plx_test_bounded_wait",)
 
@@ -106,6 +106,7 @@ def _load() -> ctypes.CDLL:
         "parallax_decode_fwd_paged": (i32, [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, f32, i32,
                                             vp, sz, i32, vp]),
         "parallax_read_probe": (i32, [vp, sz, vp, i32, i32, vp, vp]),
+        "parallax_decode_fwd_rows": (i32, [vp] * 6 + [i32] * 6 + [f32, i32, vp, sz, i32, vp, vp]),
         "plx_test_bounded_wait": (i32, [vp, ctypes.c_uint32, vp, vp]),
     }
     for name, (res, args) in sig.items():
@@ -304,6 +305,23 @@ def parallax_prefill_fwd_ex(q, r, k_cache, v_cache, seqlens, out, scale, workspa
                                         B, Hq, Hkv, D, Lq, T_max, float(scale), _out_dtype_code(out.dtype),
                                         int(p_precision), _ptr(workspace), ws_bytes, int(num_splits), _ptr(status),
                                         _stream(stream)))
+    return out
+
+
+def parallax_decode_fwd_rows(q, r, k_cache, v_cache, seqlens, out, scale, workspace=None, num_splits=0, status=None,
+                             stream=None):
+    """The keys-on-lanes tensor-core kernel for a step of up to 64 rows per KV head ((Hq / Hkv) * Lq <= 64, D = 128);
+    q, r, out [B, Hq, Lq, D]; workspace: uint8 CUDA tensor of parallax_prefill_workspace_bytes(...) bytes for split
+    records, or None for one split.  parallax_decode_fwd_multi picks this kernel by itself."""
+    _require(q, r, k_cache, v_cache, seqlens, out, workspace, status)
+    B, Hq, Lq, D = q.shape
+    Bk, Hkv, T_max, Dk = k_cache.shape
+    if Bk != B or Dk != D or tuple(out.shape) != (B, Hq, Lq, D) or tuple(r.shape) != tuple(q.shape):
+        raise ParallaxError(PLX_ERR_BAD_SHAPE)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(_lib.parallax_decode_fwd_rows(_ptr(q), _ptr(r), _ptr(k_cache), _ptr(v_cache), _ptr(seqlens), _ptr(out),
+                                         B, Hq, Hkv, D, Lq, T_max, float(scale), _out_dtype_code(out.dtype),
+                                         _ptr(workspace), ws_bytes, int(num_splits), _ptr(status), _stream(stream)))
     return out
 
 

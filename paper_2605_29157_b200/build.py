@@ -20,7 +20,7 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 SOURCES = [PKG / "csrc" / "parallax_decode.cu", PKG / "csrc" / "parallax_prefill.cu",
            PKG / "csrc" / "parallax_prepare.cu", PKG / "csrc" / "parallax_backward.cu",
-           PKG / "csrc" / "parallax_probe.cu"]
+           PKG / "csrc" / "parallax_probe.cu", PKG / "csrc" / "parallax_decode_rows.cu"]
 HEADERS = [ROOT / "include" / "parallax.h", ROOT / "include" / "parallax_test_hooks.h",
            PKG / "csrc" / "plx_common.cuh", PKG / "csrc" / "plx_tcgen05.cuh"]
 LIB = PKG / "libparallax.so"
