@@ -370,7 +370,7 @@ int parallax_decode_fwd_multi(const void* q, const void* r, const void* k_cache,
 /*
  * The same step on the tensor-core kernel that keeps the KEYS on the accumulator lanes (Algorithm 1 with
  * S^T = K_c [Q; R]^T per 128-key tile and O^T += V_c^T P^T, so the tensor work follows the rows present):
- * up to 64 rows per KV head (Lq * Hq / Hkv <= 64), D = 128, bf16 caches, contiguous layout; q, r, k_cache,
+ * up to 32 rows per KV head (Lq * Hq / Hkv <= 32), D = 128, bf16 caches, contiguous layout; q, r, k_cache,
  * v_cache, out 16-byte aligned.  Split-KV like parallax_prefill_fwd_ex: `workspace` holds split records only
  * (parallax_prefill_workspace_bytes(B, Hq, D, Lq, max_splits) bytes, 16-byte aligned; NULL = one split),
  * num_splits 0 = planned (about one CTA per SM, at least four 128-key tiles per split), records merged by the

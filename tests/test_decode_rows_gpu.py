@@ -1,5 +1,5 @@
 """GPU parity of the keys-on-lanes tensor-core kernel for multi-token decode steps (parallax_decode_fwd_rows:
-up to 64 rows per KV head) against the fp64 oracle of the multi-token causal forward."""
+up to 32 rows per KV head) against the fp64 oracle of the multi-token causal forward."""
 import numpy as np
 import pytest
 import torch
@@ -47,9 +47,80 @@ def run_rows(plx, oracle, cfg, Lq, ns=1, seqlens=None, out_dtype=torch.float32, 
     return x, out
 
 
-@pytest.mark.parametrize("G,Lq", [(2, 8), (2, 16), (2, 32), (4, 16), (1, 64), (2, 5), (4, 3), (8, 8), (1, 1), (2, 12), (3, 7)])
+@pytest.mark.parametrize("G,Lq", [(2, 8), (2, 16), (4, 8), (1, 32), (2, 5), (4, 3), (8, 4), (1, 1), (2, 12), (3, 7), (1, 16), (8, 2),
+                                  (2, 9), (5, 5)])
 @pytest.mark.parametrize("T", [128, 129, 200, 256, 1000])
 def test_rows_single_split(plx, oracle, G, Lq, T):
     """One CTA per KV head: full and ragged last tiles, the last Lq - 1 keys straddling a tile boundary."""
     cfg = wl.DecodeConfig("rows", B=2, Hq=2 * G, Hkv=2, D=128, T_max=T, seed=2100 + T + Lq)
     run_rows(plx, oracle, cfg, Lq, ns=1)
+
+
+@pytest.mark.parametrize("Lq,T,ns", [(8, 1000, 3), (16, 4096, 0), (8, 5000, 7), (12, 2048, 16), (16, 1030, 4), (10, 3000, 0),
+                                     (5, 8192, 64), (16, 640, 5)])
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_rows_split_kv(plx, oracle, Lq, T, ns, out_dtype):
+    """Split contexts (forced and planned): the split that holds the last keys gives some tokens an empty record."""
+    cfg = wl.DecodeConfig("rows split", B=3, Hq=4, Hkv=2, D=128, T_max=T, seed=2200 + T)
+    run_rows(plx, oracle, cfg, Lq, ns=ns, out_dtype=out_dtype)
+
+
+@pytest.mark.parametrize("ns", [1, 0, 6])
+def test_rows_ragged_contexts_with_poisoned_padding(plx, oracle, ns):
+    """Per-sequence lengths incl. empty, shorter than Lq, one key, tile-aligned and ragged; NaN behind every context."""
+    Lq = 12
+    cfg = wl.DecodeConfig("rows ragged", B=8, Hq=4, Hkv=2, D=128, T_max=1500, seed=2300)
+    run_rows(plx, oracle, cfg, Lq, ns=ns, seqlens=[0, 1, 5, 12, 128, 129, 1024, 1500])
+
+
+def test_rows_split_boundary_inside_the_new_tokens(plx, oracle):
+    """A split boundary that falls inside the last Lq keys: the last split holds only keys the first tokens must not see."""
+    Lq = 16
+    for T in (256 + 1, 256 + 9, 384 + 15, 512 + 3):
+        cfg = wl.DecodeConfig("rows boundary", B=2, Hq=4, Hkv=2, D=128, T_max=T, seed=2400 + T)
+        run_rows(plx, oracle, cfg, Lq, ns=(T + 127) // 128)
+
+
+@pytest.mark.parametrize("kind", ["peaked", "growing"])
+def test_rows_reference_moves_late(plx, oracle, kind):
+    """Scores that keep growing along the context (the reference exponent moves in many tiles, the accumulators are
+    rescaled in TMEM each time) and one dominant key late in the context."""
+    Lq, T = 8, 2048
+    cfg = wl.DecodeConfig("rows " + kind, B=2, Hq=4, Hkv=2, D=128, T_max=T, seed=2500)
+    x = wl.make_prefill_inputs(cfg, Lq, "cuda")
+    if kind == "peaked":
+        x["k"][:, :, 1777] = x["q"][:, ::2, 0].to(x["k"].dtype) * 3.0    # one key aligned with a query
+    else:
+        ramp = torch.linspace(0.2, 3.0, T, device="cuda").view(1, 1, T, 1)
+        x["k"] = (x["k"].float() * ramp).to(torch.bfloat16)
+    bits = {n: wl.bf16_bits(x[n]) for n in ("q", "r", "k", "v")}
+    want, _ = oracle.prefill_bf16(bits["q"], bits["r"], bits["k"], bits["v"], None, cfg.scale)
+    for ns in (1, 4):
+        ws = torch.empty(plx.parallax_prefill_workspace_bytes(cfg.B, cfg.Hq, cfg.D, Lq, 8), dtype=torch.uint8, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        out = torch.full((cfg.B, cfg.Hq, Lq, cfg.D), float("nan"), dtype=torch.float32, device="cuda")
+        plx.parallax_decode_fwd_rows(x["q"], x["r"], x["k"], x["v"], None, out, cfg.scale, ws, ns, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert_parity(out.cpu().numpy(), want, torch.float32, f"{kind} ns={ns}")
+
+
+def test_rows_rejects_what_it_does_not_serve(plx):
+    q = torch.zeros(1, 4, 40, 128, dtype=torch.bfloat16, device="cuda")      # 80 rows per KV head
+    k = torch.zeros(1, 2, 256, 128, dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros(1, 4, 40, 128, dtype=torch.float32, device="cuda")
+    with pytest.raises(plx.ParallaxError) as e:
+        plx.parallax_decode_fwd_rows(q, q, k, k, None, out, 0.1)
+    assert e.value.status == plx.PLX_ERR_UNSUPPORTED
+    q = torch.zeros(1, 4, 4, 64, dtype=torch.bfloat16, device="cuda")        # head dimension 64
+    k = torch.zeros(1, 2, 256, 64, dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros(1, 4, 4, 64, dtype=torch.float32, device="cuda")
+    with pytest.raises(plx.ParallaxError) as e:
+        plx.parallax_decode_fwd_rows(q, q, k, k, None, out, 0.1)
+    assert e.value.status == plx.PLX_ERR_UNSUPPORTED
+    q = torch.zeros(1, 4, 4, 128, dtype=torch.bfloat16, device="cuda")
+    k = torch.zeros(1, 2, 256, 128, dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros(1, 4, 4, 128, dtype=torch.float32, device="cuda")
+    with pytest.raises(plx.ParallaxError) as e:                                # splits without room for records
+        plx.parallax_decode_fwd_rows(q, q, k, k, None, out, 0.1, None, 3)
+    assert e.value.status == plx.PLX_ERR_WORKSPACE
