@@ -33,6 +33,13 @@
 #include "parallax.h"
 #include "plx_common.cuh"
 
+// Defined in parallax_decode_rows.cu: multi-token decode steps of up to 32 rows per KV head on the tensor cores with
+// the keys on the accumulator lanes.
+bool plx_decode_rows_supported(int Hq, int Hkv, int D, int Lq);
+int plx_decode_rows_fwd(const void* q, const void* r, const void* k_cache, const void* v_cache, const int32_t* seqlens,
+                        void* out, int B, int Hq, int Hkv, int D, int Lq, int T_max, float scale, int out_dtype,
+                        void* records, size_t record_bytes, int num_splits, int32_t* status, cudaStream_t stream);
+
 namespace {
 
 // Compile-time tuning knobs (defaults are the measured best on B200).
@@ -1763,6 +1770,22 @@ int parallax_decode_fwd_multi(const void* q, const void* r, const void* k_cache,
 {
     if (Lq <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || B <= 0) return PLX_ERR_BAD_SHAPE;
     if (workspace && !aligned(workspace, 16)) return PLX_ERR_ALIGNMENT;
+    // Nine to 32 rows per KV head at D = 128: the tensor-core kernel with the keys on the accumulator lanes, whose work
+    // follows the rows present.  Measured against the routes below (8 KV heads, 10 / 16 / 24 / 32 rows, us per step):
+    // 64 x 8192 keys 342 / 352 / 412 / 462 against 474 / 506 / 722 / 766; 16 x 8192 94 / 92 / 107 / 108 against 146 / 154 /
+    // 182 / 182; 8 x 8192 56 / 56 / 78 / 72 against 80 / 87 / 116 / 107; 2 x 131072 166 / 164 / 188 / 202 against 323 / 334 /
+    // 339 / 339; 1 x 32768 36 / 37 / 44 / 45 against 52 / 59 / 57 / 58.  (Up to eight rows the decode kernel stays ahead
+    // or level at large batches: 64 x 8192, 2 / 4 / 8 rows: 298 / 300 / 314 against 324 / 329 / 340.)
+    if (static_cast<long long>(Hq / Hkv) * Lq > kMultiTokenDecodeRows && plx_decode_rows_supported(Hq, Hkv, D, Lq) &&
+        aligned(q, 16) && aligned(r, 16) && aligned(out, 16) && aligned(k_cache, 16) && aligned(v_cache, 16)) {
+        void* rec = nullptr;
+        size_t rec_bytes = 0;
+        records_region(workspace, workspace_bytes, B, Hq * Lq, D, &rec, &rec_bytes);
+        int32_t* status = (workspace && workspace_bytes >= kHeaderBytes) ? static_cast<int32_t*>(workspace) : nullptr;
+        return plx_decode_rows_fwd(q, r, k_cache, v_cache, seqlens, out, B, Hq, Hkv, D, Lq, T_max, scale, out_dtype, rec,
+                                   rec_bytes, rec ? num_splits : (num_splits > 1 ? 1 : num_splits), status,
+                                   static_cast<cudaStream_t>(stream));
+    }
     if (use_tensor_core_kernel(q, r, out, B, Hq, Hkv, Lq, D)) {
         void* rec = nullptr;
         size_t rec_bytes = 0;
