@@ -36,9 +36,11 @@
 // Defined in parallax_decode_rows.cu: multi-token decode steps of up to 32 rows per KV head on the tensor cores with
 // the keys on the accumulator lanes.
 bool plx_decode_rows_supported(int Hq, int Hkv, int D, int Lq);
+bool plx_decode_rows_page_size_ok(int page_size);
 int plx_decode_rows_fwd(const void* q, const void* r, const void* k_cache, const void* v_cache, const int32_t* seqlens,
                         void* out, int B, int Hq, int Hkv, int D, int Lq, int T_max, float scale, int out_dtype,
-                        void* records, size_t record_bytes, int num_splits, int32_t* status, cudaStream_t stream);
+                        void* records, size_t record_bytes, int num_splits, int32_t* status, cudaStream_t stream,
+                        const int32_t* block_table, int page_size, int max_pages, long long pool_rows);
 
 namespace {
 
@@ -1784,7 +1786,7 @@ int parallax_decode_fwd_multi(const void* q, const void* r, const void* k_cache,
         int32_t* status = (workspace && workspace_bytes >= kHeaderBytes) ? static_cast<int32_t*>(workspace) : nullptr;
         return plx_decode_rows_fwd(q, r, k_cache, v_cache, seqlens, out, B, Hq, Hkv, D, Lq, T_max, scale, out_dtype, rec,
                                    rec_bytes, rec ? num_splits : (num_splits > 1 ? 1 : num_splits), status,
-                                   static_cast<cudaStream_t>(stream));
+                                   static_cast<cudaStream_t>(stream), nullptr, 0, 0, 0);
     }
     if (use_tensor_core_kernel(q, r, out, B, Hq, Hkv, Lq, D)) {
         void* rec = nullptr;
@@ -1875,6 +1877,20 @@ int parallax_decode_fwd_multi_paged(const void* q, const void* r, const void* k_
     if (workspace && !aligned(workspace, 16)) return PLX_ERR_ALIGNMENT;
     if (num_pages <= 0 || page_size <= 0 || page_size % kTileKeys != 0 || max_pages_per_seq <= 0)
         return PLX_ERR_BAD_SHAPE;
+    if (static_cast<long long>(Hq / Hkv) * Lq > kMultiTokenDecodeRows && plx_decode_rows_supported(Hq, Hkv, D, Lq) &&
+        plx_decode_rows_page_size_ok(page_size) && aligned(q, 16) && aligned(r, 16) && aligned(out, 16) &&
+        aligned(k_pages, 16) && aligned(v_pages, 16)) {  // nine to 32 rows per KV head: as in parallax_decode_fwd_multi
+        const long long T_cap = static_cast<long long>(page_size) * max_pages_per_seq;
+        const long long pool = static_cast<long long>(num_pages) * Hkv * page_size;
+        if (T_cap >= (1LL << 31) - 65536 || pool >= (1LL << 31) - 65536) return PLX_ERR_BAD_SHAPE;
+        void* rec = nullptr;
+        size_t rec_bytes = 0;
+        records_region(workspace, workspace_bytes, B, Hq * Lq, D, &rec, &rec_bytes);
+        int32_t* status = (workspace && workspace_bytes >= kHeaderBytes) ? static_cast<int32_t*>(workspace) : nullptr;
+        return plx_decode_rows_fwd(q, r, k_pages, v_pages, seqlens, out, B, Hq, Hkv, D, Lq, static_cast<int>(T_cap), scale,
+                                   out_dtype, rec, rec_bytes, rec ? num_splits : (num_splits > 1 ? 1 : num_splits), status,
+                                   static_cast<cudaStream_t>(stream), block_table, page_size, max_pages_per_seq, pool);
+    }
     if (page_size % 64 == 0 && use_tensor_core_kernel(q, r, out, B, Hq, Hkv, Lq, D)) {  // that kernel walks 64-key tiles
         void* rec = nullptr;
         size_t rec_bytes = 0;

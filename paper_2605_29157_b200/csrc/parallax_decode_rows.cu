@@ -29,6 +29,10 @@
 int plx_combine_after_producer(const float* partials, void* out, int rows, int D, int num_splits, int out_dtype,
                                cudaStream_t stream);
 
+#ifndef PLX_DEBUG_CHECKS
+#define PLX_DEBUG_CHECKS 0  // 1: page ids are verified against the pool before they are followed
+#endif
+
 namespace {
 
 constexpr int BK = 128;  // keys per tile = TMEM lanes
@@ -53,7 +57,7 @@ template <int NR>
 struct RowsCfg {
     static_assert(NR == 16 || NR == 32, "rows per KV head");
     static constexpr int RPT = NR / 2;                    // rows per element-wise thread
-    static constexpr int kStagesK = 3, kStagesV = NR == 16 ? 3 : 2;
+    static constexpr int kStagesK = NR == 16 ? 3 : 2, kStagesV = 3;
     static constexpr int kBoxQR = 2 * NR * 128;           // [Q rows; R rows] x 64 columns: the N = 2 NR operand of the score product
     static constexpr int kTileQR = 2 * kBoxQR;
     static constexpr int kPBlocks = 4 * NR / 64;          // 64-wide blocks of [P1 | P1 res | P2 | P2 res]
@@ -85,6 +89,11 @@ struct RowsParams {
     int num_splits, tiles_per_split;
     float scale_log2e;
     int out_dtype;
+    // paged cache: int32 [B, max_pages] page ids (else nullptr); pools [num_pages, Hkv, page_size, D]; page_size
+    // divides 128 or is a multiple of it, so a 128-key tile is a whole number of boxes of `page_box` keys
+    const int32_t* block_table;
+    int page_size, max_pages, page_box;
+    long long pool_rows;
 };
 
 __device__ __forceinline__ void ew_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kEwThreads) : "memory"); }
@@ -237,19 +246,56 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 tma_load_2d(base + C::kOffQR + h * C::kBoxQR, &tmQ, bar(kBarQR), 64 * h, static_cast<int>(row0));
                 tma_load_2d(base + C::kOffQR + h * C::kBoxQR + NR * 128, &tmR, bar(kBarQR), 64 * h, static_cast<int>(row0));
             }
+            const int32_t* const table = p.block_table ? p.block_table + static_cast<size_t>(b) * p.max_pages : nullptr;
             for (int j = 0; j < n_tiles; ++j) {
                 const int sk = j % C::kStagesK, sv = j % C::kStagesV;
-                const int krow = static_cast<int>(kv_row0) + (jt0 + j) * BK;
+                const int key0 = (jt0 + j) * BK;
                 if (j >= C::kStagesK) wait_or_flag(bar(kBarKFree + sk), (j / C::kStagesK - 1) & 1, p.status);
-                mbar_expect_tx(bar(kBarKFull + sk), kTileKV);
+                if (!table) {
+                    const int krow = static_cast<int>(kv_row0) + key0;
+                    mbar_expect_tx(bar(kBarKFull + sk), kTileKV);
 #pragma unroll
-                for (int h = 0; h < 2; ++h)
-                    tma_load_2d(base + C::kOffK + sk * kTileKV + h * kBoxKV, &tmK, bar(kBarKFull + sk), 64 * h, krow);
-                if (j >= C::kStagesV) wait_or_flag(bar(kBarVFree + sv), (j / C::kStagesV - 1) & 1, p.status);
-                mbar_expect_tx(bar(kBarVFull + sv), kTileKV);
+                    for (int h = 0; h < 2; ++h)
+                        tma_load_2d(base + C::kOffK + sk * kTileKV + h * kBoxKV, &tmK, bar(kBarKFull + sk), 64 * h, krow);
+                    if (j >= C::kStagesV) wait_or_flag(bar(kBarVFree + sv), (j / C::kStagesV - 1) & 1, p.status);
+                    mbar_expect_tx(bar(kBarVFull + sv), kTileKV);
 #pragma unroll
-                for (int h = 0; h < 2; ++h)
-                    tma_load_2d(base + C::kOffV + sv * kTileKV + h * kBoxKV, &tmV, bar(kBarVFull + sv), 64 * h, krow);
+                    for (int h = 0; h < 2; ++h)
+                        tma_load_2d(base + C::kOffV + sv * kTileKV + h * kBoxKV, &tmV, bar(kBarVFull + sv), 64 * h, krow);
+                } else {
+                    // Paged: the tile is fetched in boxes of page_box keys, each from its page.  Boxes that lie wholly
+                    // past the context are not fetched (their pages need not exist): those rows of the tile keep what
+                    // an earlier tile left there, their scores are masked and their V rows are cleared before use.
+                    const int pb = p.page_box;
+                    const int nbox = min(BK / pb, (L - key0 + pb - 1) / pb);
+                    int rows_of[BK / 16];
+                    for (int i = 0; i < nbox; ++i) {
+                        const int key = key0 + i * pb;
+                        const int pg = key / p.page_size;
+                        int id = __ldg(table + pg);
+#if PLX_DEBUG_CHECKS
+                        if (id < 0 || (static_cast<long long>(id) * p.Hkv + hkv + 1) * p.page_size > p.pool_rows) {
+                            if (p.status) atomicExch(p.status, PLX_ERR_DEVICE_CHECK);  // a page id outside the pool: not followed
+                            id = 0;
+                        }
+#endif
+                        rows_of[i] = (id * p.Hkv + hkv) * p.page_size + (key - pg * p.page_size);
+                    }
+                    const uint32_t bytes = static_cast<uint32_t>(nbox) * pb * 128 * 2;
+                    mbar_expect_tx(bar(kBarKFull + sk), bytes);
+                    for (int i = 0; i < nbox; ++i)
+#pragma unroll
+                        for (int h = 0; h < 2; ++h)
+                            tma_load_2d(base + C::kOffK + sk * kTileKV + h * kBoxKV + i * pb * 128, &tmK, bar(kBarKFull + sk),
+                                        64 * h, rows_of[i]);
+                    if (j >= C::kStagesV) wait_or_flag(bar(kBarVFree + sv), (j / C::kStagesV - 1) & 1, p.status);
+                    mbar_expect_tx(bar(kBarVFull + sv), bytes);
+                    for (int i = 0; i < nbox; ++i)
+#pragma unroll
+                        for (int h = 0; h < 2; ++h)
+                            tma_load_2d(base + C::kOffV + sv * kTileKV + h * kBoxKV + i * pb * 128, &tmV, bar(kBarVFull + sv),
+                                        64 * h, rows_of[i]);
+                }
             }
         }
         __syncwarp();
@@ -554,16 +600,23 @@ bool plx_decode_rows_supported(int Hq, int Hkv, int D, int Lq)
 }
 
 // q, r, out [B, Hq, Lq, D]; `records` / `record_bytes`: room for split records (may be null: one split).
+// Paged cache: block_table != nullptr, k_cache / v_cache are the page pools of pool_rows rows, T_max = page_size * max_pages.
+bool plx_decode_rows_page_size_ok(int page_size) { return page_size > 0 && page_size % 16 == 0 && (BK % page_size == 0 || page_size % BK == 0); }
+
 int plx_decode_rows_fwd(const void* q, const void* r, const void* k_cache, const void* v_cache, const int32_t* seqlens,
                         void* out, int B, int Hq, int Hkv, int D, int Lq, int T_max, float scale, int out_dtype,
-                        void* records, size_t record_bytes, int num_splits, int32_t* status, cudaStream_t stream)
+                        void* records, size_t record_bytes, int num_splits, int32_t* status, cudaStream_t stream,
+                        const int32_t* block_table, int page_size, int max_pages, long long pool_rows)
 {
     if (!q || !r || !k_cache || !v_cache || !out) return PLX_ERR_NULL_POINTER;
     if (B <= 0 || Hq <= 0 || Hkv <= 0 || Lq <= 0 || T_max <= 0 || Hq % Hkv != 0) return PLX_ERR_BAD_SHAPE;
     if (!plx_decode_rows_supported(Hq, Hkv, D, Lq)) return PLX_ERR_UNSUPPORTED;
+    if (block_table && (!plx_decode_rows_page_size_ok(page_size) || max_pages <= 0 || pool_rows <= 0)) return PLX_ERR_UNSUPPORTED;
     if (out_dtype != PLX_OUT_BF16 && out_dtype != PLX_OUT_F32) return PLX_ERR_BAD_SHAPE;
     if (num_splits < 0 || num_splits > PLX_MAX_SPLITS) return PLX_ERR_BAD_SHAPE;
-    const long long q_rows = static_cast<long long>(B) * Hq * Lq, kv_rows = static_cast<long long>(B) * Hkv * T_max;
+    const long long q_rows = static_cast<long long>(B) * Hq * Lq;
+    const long long kv_rows = block_table ? pool_rows : static_cast<long long>(B) * Hkv * T_max;
+    const int page_box = block_table ? (page_size < BK ? page_size : BK) : BK;
     if (q_rows >= (1LL << 31) - 65536 || kv_rows >= (1LL << 31) - 65536) return PLX_ERR_BAD_SHAPE;
     if (!plx_aligned(q, 16) || !plx_aligned(r, 16) || !plx_aligned(k_cache, 16) || !plx_aligned(v_cache, 16) ||
         !plx_aligned(out, 16) || (records && !plx_aligned(records, 16)))
@@ -576,8 +629,8 @@ int plx_decode_rows_fwd(const void* q, const void* r, const void* k_cache, const
     const CUtensorMapL2promotion promo = CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
     if ((rc = make_tensor_map_2d(&tmQ, q, D, static_cast<uint64_t>(q_rows), nr, promo)) != PLX_OK) return rc;
     if ((rc = make_tensor_map_2d(&tmR, r, D, static_cast<uint64_t>(q_rows), nr, promo)) != PLX_OK) return rc;
-    if ((rc = make_tensor_map_2d(&tmK, k_cache, D, static_cast<uint64_t>(kv_rows), BK, promo)) != PLX_OK) return rc;
-    if ((rc = make_tensor_map_2d(&tmV, v_cache, D, static_cast<uint64_t>(kv_rows), BK, promo)) != PLX_OK) return rc;
+    if ((rc = make_tensor_map_2d(&tmK, k_cache, D, static_cast<uint64_t>(kv_rows), page_box, promo)) != PLX_OK) return rc;
+    if ((rc = make_tensor_map_2d(&tmV, v_cache, D, static_cast<uint64_t>(kv_rows), page_box, promo)) != PLX_OK) return rc;
 
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -618,7 +671,7 @@ int plx_decode_rows_fwd(const void* q, const void* r, const void* k_cache, const
     ns = (tiles_max + tps - 1) / tps;  // no split without a tile
     if (base_ctas * ns > 0x7fffffffLL) return PLX_ERR_BAD_SHAPE;
     RowsParams rp{seqlens, out, ns > 1 ? static_cast<float*>(records) : nullptr, status, B, Hq, Hkv, Lq, T_max,
-                  rows, ns, tps, scale * 1.4426950408889634f, out_dtype};
+                  rows, ns, tps, scale * 1.4426950408889634f, out_dtype, block_table, page_size, max_pages, page_box, pool_rows};
     PlxNvtxRange nvtx_range("plx_decode_rows_fwd");
     const unsigned grid = static_cast<unsigned>(base_ctas * ns);
     rc = nr == 16 ? launch_rows<16>(tmQ, tmR, tmK, tmV, rp, grid, dev, stream)
@@ -636,5 +689,5 @@ extern "C" int parallax_decode_fwd_rows(const void* q, const void* r, const void
                                         int num_splits, int32_t* status, void* stream)
 {
     return plx_decode_rows_fwd(q, r, k_cache, v_cache, seqlens, out, B, Hq, Hkv, D, Lq, T_max, scale, out_dtype, workspace,
-                               workspace_bytes, num_splits, status, static_cast<cudaStream_t>(stream));
+                               workspace_bytes, num_splits, status, static_cast<cudaStream_t>(stream), nullptr, 0, 0, 0);
 }

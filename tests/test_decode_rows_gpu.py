@@ -124,3 +124,38 @@ def test_rows_rejects_what_it_does_not_serve(plx):
     with pytest.raises(plx.ParallaxError) as e:                                # splits without room for records
         plx.parallax_decode_fwd_rows(q, q, k, k, None, out, 0.1, None, 3)
     assert e.value.status == plx.PLX_ERR_WORKSPACE
+
+
+@pytest.mark.parametrize("page_size", [16, 32, 64, 128, 256, 48])
+@pytest.mark.parametrize("Lq,ns", [(6, 1), (12, 0), (16, 5)])
+def test_rows_over_a_paged_cache(plx, oracle, page_size, Lq, ns):
+    """parallax_decode_fwd_multi_paged at 12 to 32 rows per KV head: page sizes that divide the 128-key tile or are a
+    multiple of it go to the keys-on-lanes kernel (a tile fetched page by page), 48 takes the older routes; random page
+    order, NaN in unused pages and page tails, ragged contexts incl. one shorter than Lq + a page."""
+    T = 1536
+    cfg = wl.DecodeConfig("rows paged", B=4, Hq=4, Hkv=2, D=128, T_max=T, ragged=(Lq, T), seed=2600 + page_size)
+    x = wl.make_prefill_inputs(cfg, Lq, "cuda")
+    kp, vp, table = wl.to_paged(x["k"], x["v"], page_size, seed=9)
+    out = torch.full((cfg.B, cfg.Hq, Lq, cfg.D), float("nan"), dtype=torch.float32, device="cuda")
+    ws = plx.alloc_workspace(cfg.B, cfg.Hq * Lq, cfg.D, plx.PLX_MAX_SPLITS if ns == 0 else ns, "cuda")
+    plx.parallax_decode_fwd_multi_paged(x["q"], x["r"], kp, vp, table, x["seqlens"], out, cfg.scale, ws, ns)
+    torch.cuda.synchronize()
+    assert plx.parallax_workspace_status(ws) == 0
+    bits = {n: wl.bf16_bits(x[n]) for n in ("q", "r", "k", "v")}
+    want, _ = oracle.prefill_bf16(bits["q"], bits["r"], bits["k"], bits["v"], x["seqlens_host"], cfg.scale)
+    assert_parity(out.cpu().numpy(), want, torch.float32, f"rows paged ps={page_size} Lq={Lq}")
+
+
+def test_multi_query_group_of_sixteen_in_one_token_steps(plx, oracle):
+    """One token, sixteen and 24 query heads per KV head: parallax_decode_fwd_ex hands the step to the keys-on-lanes kernel."""
+    for G in (16, 24):
+        cfg = wl.DecodeConfig("mqa rows", B=3, Hq=2 * G, Hkv=2, D=128, T_max=2100, ragged=(1, 2100), seed=2700 + G)
+        x = wl.make_inputs(cfg, "cuda", poison_padding=True)
+        from parity_util import oracle_full
+        want = oracle_full(oracle, x, cfg.scale, x["seqlens_host"])
+        out = torch.full((cfg.B, cfg.Hq, cfg.D), float("nan"), dtype=torch.float32, device="cuda")
+        ws = plx.alloc_workspace(cfg.B, cfg.Hq, cfg.D, plx.PLX_MAX_SPLITS, "cuda")
+        plx.parallax_decode_fwd_ex(x["q"], x["r"], x["k"], x["v"], x["seqlens"], out, cfg.scale, ws, 0)
+        torch.cuda.synchronize()
+        assert plx.parallax_workspace_status(ws) == 0
+        assert_parity(out.cpu().numpy(), want, torch.float32, f"G={G}")

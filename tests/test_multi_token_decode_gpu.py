@@ -151,12 +151,14 @@ def test_multi_token_paged_cache(plx, oracle, page_size, Lq, T, ns):
     assert_parity(out.cpu().numpy(), want, torch.float32, f"multi paged ps={page_size}")
 
 
+@pytest.mark.parametrize("D", [64, 128])
 @pytest.mark.parametrize("G,Lq", [(2, 5), (2, 6), (2, 8), (4, 4), (2, 7)])
-def test_ten_to_sixteen_rows_stay_on_the_decode_kernel(plx, oracle, G, Lq):
-    """10 / 12 / 16 rows per KV head are served by two CTAs of the decode kernel (five to eight rows each)
-    instead of the tensor-core kernel; 14 rows likewise (2 x 7).  Ragged contexts, NaN padding, planned splits."""
+def test_ten_to_sixteen_rows(plx, oracle, D, G, Lq):
+    """10 / 12 / 14 / 16 rows per KV head: at D = 64 two CTAs of the decode kernel (five to eight rows each), at
+    D = 128 the keys-on-lanes tensor-core kernel (the options-struct entry stays on the decode kernel either way).
+    Ragged contexts, NaN padding, planned splits."""
     B, Hkv = 16, 8
-    cfg = wl.DecodeConfig("two-cta rows", B=B, Hq=Hkv * G, Hkv=Hkv, D=128, T_max=700, seed=1700 + G * Lq)
+    cfg = wl.DecodeConfig("ten to sixteen rows", B=B, Hq=Hkv * G, Hkv=Hkv, D=D, T_max=700, seed=1700 + G * Lq)
     g = np.random.default_rng(G * 100 + Lq)
     lens = g.integers(Lq, 701, size=B)
     lens[0], lens[1] = 700, Lq
