@@ -431,7 +431,9 @@ def run_ours(args, rank, world, local_rank):
     t_call = timer.run(step, args.steps)
     ms_per_step = t_call["ms_per_step"]
     # one launch per call, except steps the library hands to the tensor-core kernel (more than eight rows per KV head)
-    launches_per_step = tensor_core_launches(cfg, Lq, sms) if routed_to_tensor_core(cfg, Lq) and not (args.fp8_kv or args.page_size) else 1
+    route = "decode" if args.fp8_kv else multi_token_route(cfg, Lq, args.page_size)
+    launches_per_step = (rows_kernel_launches(cfg, Lq, sms) if route == "rows" else
+                         tensor_core_launches(cfg, Lq, sms) if route == "row-major" and not args.page_size else 1)
     value = whole_job_value(kv_bytes, world, ms_per_step)
     assert plx.parallax_workspace_status(ws) == 0, "device-side wait timed out"
     us_graph = graph_replay_us(step, nsets)
@@ -458,7 +460,9 @@ def run_ours(args, rank, world, local_rank):
     achieved = kv_bytes / (ms_kernel * 1e-3) / 1e9
     traffic, traffic_src = ((None, None) if (args.page_size or Lq > 1 or args.batch or args.splits) else
                             ncu_traffic(cfg.name, args.fp8_kv))
-    roofline = {"bound": "hbm", "kernel": "plx_decode_kernel", "achieved": round(achieved, 1), "peak": peak,
+    roofline = {"bound": "hbm", "kernel": {"decode": "plx_decode_kernel", "rows": "plx_decode_rows_kernel",
+                                           "row-major": "plx_prefill_kernel"}[route],
+                "achieved": round(achieved, 1), "peak": peak,
                 "peak_source": f"{peak_src} copy bandwidth (read + write)", "unit": "GB/s", "frac": round(achieved / peak, 4),
                 "frac_of_8TBps_nominal": round(achieved / 8000.0, 4),
                 "us_per_launch": round(ms_kernel * 1e3, 2),
@@ -544,18 +548,43 @@ def run_ours(args, rank, world, local_rank):
     return result
 
 
-def routed_to_tensor_core(cfg, Lq):
-    """Mirrors the library's routing of a multi-token step (only to count launches): up to eight rows per KV head
-    run on the decode kernel, nine to sixteen too when they split into two CTAs of at most eight rows, everything
-    else on the tensor-core kernel."""
+def multi_token_route(cfg, Lq, page_size=0):
+    """Mirrors the library's routing of a multi-token step (only to name the kernel and count launches): up to
+    eight rows per KV head the decode kernel; nine to 32 rows at D = 128 the keys-on-lanes tensor-core kernel
+    ("rows"; paged caches when the page size divides 128 or is a multiple of it); otherwise nine to sixteen rows
+    that split into two CTAs of at most eight stay on the decode kernel and everything else goes to the row-major
+    tensor-core kernel."""
     rows = cfg.G * Lq
     if rows <= 8:
-        return False
+        return "decode"
+    if rows <= 32 and cfg.D == 128 and (not page_size or 128 % page_size == 0 or page_size % 128 == 0):
+        return "rows"
     if rows <= 16:
         g = max(c for c in range(1, 9) if rows % c == 0)
         if rows // g <= 2:
-            return False
-    return True
+            return "decode"
+    return "row-major"
+
+
+def routed_to_tensor_core(cfg, Lq):
+    return multi_token_route(cfg, Lq) != "decode"
+
+
+def rows_kernel_launches(cfg, Lq, sms):
+    """Launches per call of the keys-on-lanes kernel: 2 when the library splits the keys (kernel + merge), else 1.
+    Mirrors the library's plan only to count launches."""
+    base, tiles = cfg.B * cfg.Hkv, -(-cfg.T_max // 128)
+    if base < sms:
+        ns = min(sms // base, max(1, tiles // 4), 64)
+    else:
+        ns, best = 1, 1e30
+        for c in range(1, 5):
+            if tiles // c < 16:
+                break
+            cost = -(-base * c // sms) / c * (1.0 + 0.02 * (c - 1))
+            if cost < best - 1e-9:
+                best, ns = cost, c
+    return 2 if ns > 1 else 1
 
 
 def tensor_core_launches(cfg, Lq, sms):

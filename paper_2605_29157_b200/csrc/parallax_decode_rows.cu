@@ -33,15 +33,37 @@ int plx_combine_after_producer(const float* partials, void* out, int rows, int D
 #define PLX_DEBUG_CHECKS 0  // 1: page ids are verified against the pool before they are followed
 #endif
 
+// Cycle accounting for experiments (-DPLX_TRACE=1; never part of the shipped build): CTA 0 accumulates the cycles
+// its element-wise thread 0, its issuing thread and its producer thread spend in each phase of a tile.
+#ifndef PLX_TRACE
+#define PLX_TRACE 0
+#endif
+#if PLX_TRACE
+__device__ long long g_rows_trace[32];
+#define ROWS_T0 long long tr_t = clock64(), tr_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}
+#define ROWS_T(i)                           \
+    do {                                    \
+        const long long tr_now = clock64(); \
+        tr_acc[(i) & 7] += tr_now - tr_t;   \
+        tr_t = tr_now;                      \
+    } while (0)
+#define ROWS_FLUSH(base_index)                                                    \
+    do {                                                                          \
+        if (blockIdx.x == 0)                                                      \
+            for (int tr_i = 0; tr_i < 8; ++tr_i) g_rows_trace[(base_index) + tr_i] = tr_acc[tr_i]; \
+    } while (0)
+#else
+#define ROWS_T0
+#define ROWS_T(i)
+#define ROWS_FLUSH(base_index)
+#endif
+
 namespace {
 
 constexpr int BK = 128;  // keys per tile = TMEM lanes
 constexpr int HD = 128;  // head dimension
 constexpr int kMaxRows = 32;
-constexpr int kEwWarps = 8;                    // element-wise warps: two threads per key, half of the rows each
-constexpr int kEwThreads = kEwWarps * 32;
-constexpr int kMmaWarp = kEwWarps, kTmaWarp = kEwWarps + 1;
-constexpr int kRowsThreads = (kEwWarps + 2) * 32;
+constexpr int kRowsPerThread = 8;              // rows per element-wise thread: NR / 8 threads share a key
 constexpr int kBoxKV = BK * 128;       // [128 keys x 64 columns] bf16 box: 16 KiB
 constexpr int kTileKV = 2 * kBoxKV;    // K or V tile
 constexpr int kBlockP = BK * 128;      // [128 keys x 64 columns of the stacked weights] bf16: 16 KiB
@@ -56,7 +78,12 @@ constexpr int REC = 2 * HD + 4;
 template <int NR>
 struct RowsCfg {
     static_assert(NR == 16 || NR == 32, "rows per KV head");
-    static constexpr int RPT = NR / 2;                    // rows per element-wise thread
+    static constexpr int RPT = kRowsPerThread;
+    static constexpr int kParts = NR / RPT;               // element-wise threads per key (2 or 4)
+    static constexpr int kEwWarps = 4 * kParts;           // four warps cover the 128 keys (TMEM lanes) of a tile
+    static constexpr int kEwThreads = kEwWarps * 32;
+    static constexpr int kMmaWarp = kEwWarps, kTmaWarp = kEwWarps + 1;
+    static constexpr int kThreads = (kEwWarps + 2) * 32;
     static constexpr int kStagesK = NR == 16 ? 3 : 2, kStagesV = 3;
     static constexpr int kBoxQR = 2 * NR * 128;           // [Q rows; R rows] x 64 columns: the N = 2 NR operand of the score product
     static constexpr int kTileQR = 2 * kBoxQR;
@@ -70,7 +97,7 @@ struct RowsCfg {
     static constexpr int kOffTmemSlot = kOffBar + kNumBars * 8;
     static constexpr int kOffRef = kOffTmemSlot + 16;     // float [NR]: reference exponent of each row (log2 units)
     static constexpr int kOffAlpha = kOffRef + NR * 4;    // float [NR]: rescale factors of a tile that moves references
-    static constexpr int kOffWmax = kOffAlpha + NR * 4;   // float [8 warps][RPT]: per-warp tile maxima
+    static constexpr int kOffWmax = kOffAlpha + NR * 4;   // float [element-wise warps][RPT]: per-warp tile maxima
     static constexpr int kSmemBytes = kOffWmax + kEwWarps * RPT * 4;
     static_assert(kSmemBytes <= 232448, "shared-memory budget of one CTA");
     static_assert(kOffK % 1024 == 0 && kOffBar % 8 == 0, "alignment of the tiles and barriers");
@@ -96,8 +123,10 @@ struct RowsParams {
     long long pool_rows;
 };
 
+template <int kEwThreads>
 __device__ __forceinline__ void ew_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kEwThreads) : "memory"); }
 // barrier among the element-wise warps that also ORs a predicate over them
+template <int kEwThreads>
 __device__ __forceinline__ bool ew_barrier_or(bool pred)
 {
     uint32_t r;
@@ -133,18 +162,8 @@ __device__ __forceinline__ float warp_transpose_reduce(float (&v)[N], int lane)
     return v[0];
 }
 
-template <int N>
-__device__ __forceinline__ void ld_cols(uint32_t taddr, uint32_t (&r)[N])
-{
-    if constexpr (N == 8) tmem_ld8(taddr, r);
-    else tmem_ld16(taddr, r);
-}
-template <int N>
-__device__ __forceinline__ void st_cols(uint32_t taddr, const uint32_t (&r)[N])
-{
-    if constexpr (N == 8) tmem_st8(taddr, r);
-    else tmem_st16(taddr, r);
-}
+__device__ __forceinline__ void ld_cols(uint32_t taddr, uint32_t (&r)[8]) { tmem_ld8(taddr, r); }
+__device__ __forceinline__ void st_cols(uint32_t taddr, const uint32_t (&r)[8]) { tmem_st8(taddr, r); }
 
 __device__ __forceinline__ void store_value(void* out, size_t idx, float v, int out_dtype)
 {
@@ -162,13 +181,14 @@ __device__ __forceinline__ void store_value(void* out, size_t idx, float v, int 
 // buffer), the weight tiles are single (P full <-> P.V done hand over one tile at a time), the K and V rings
 // have a full / free pair per stage.
 template <int NR>
-__global__ void __launch_bounds__(kRowsThreads, 1)
+__global__ void __launch_bounds__(RowsCfg<NR>::kThreads, 1)
 plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmR,
                        const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                        const RowsParams p)
 {
     using C = RowsCfg<NR>;
-    constexpr int RPT = C::RPT;
+    constexpr int RPT = C::RPT, kEwWarps = C::kEwWarps, kEwThreads = C::kEwThreads, kMmaWarp = C::kMmaWarp,
+                  kTmaWarp = C::kTmaWarp, kRowsThreads = C::kThreads;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t base = smem_u32(smem_raw);
     uint8_t* const smem = smem_raw;
@@ -247,17 +267,22 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 tma_load_2d(base + C::kOffQR + h * C::kBoxQR + NR * 128, &tmR, bar(kBarQR), 64 * h, static_cast<int>(row0));
             }
             const int32_t* const table = p.block_table ? p.block_table + static_cast<size_t>(b) * p.max_pages : nullptr;
+            ROWS_T0;
             for (int j = 0; j < n_tiles; ++j) {
                 const int sk = j % C::kStagesK, sv = j % C::kStagesV;
                 const int key0 = (jt0 + j) * BK;
+                ROWS_T(18);
                 if (j >= C::kStagesK) wait_or_flag(bar(kBarKFree + sk), (j / C::kStagesK - 1) & 1, p.status);
+                ROWS_T(16);
                 if (!table) {
                     const int krow = static_cast<int>(kv_row0) + key0;
                     mbar_expect_tx(bar(kBarKFull + sk), kTileKV);
 #pragma unroll
                     for (int h = 0; h < 2; ++h)
                         tma_load_2d(base + C::kOffK + sk * kTileKV + h * kBoxKV, &tmK, bar(kBarKFull + sk), 64 * h, krow);
+                    ROWS_T(18);
                     if (j >= C::kStagesV) wait_or_flag(bar(kBarVFree + sv), (j / C::kStagesV - 1) & 1, p.status);
+                    ROWS_T(17);
                     mbar_expect_tx(bar(kBarVFull + sv), kTileKV);
 #pragma unroll
                     for (int h = 0; h < 2; ++h)
@@ -297,6 +322,7 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                                         64 * h, rows_of[i]);
                 }
             }
+            ROWS_FLUSH(16);
         }
         __syncwarp();
     } else if (warp == kMmaWarp) {
@@ -306,10 +332,14 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         const uint64_t dQR = make_smem_desc(base + C::kOffQR, 0, 1024);
         const uint64_t dP = make_smem_desc(base + C::kOffP, kBlockP, 1024);
         wait_or_flag(bar(kBarQR), 0, p.status);
+        ROWS_T0;
         auto score = [&](int j) {
             const int s = j & 1, sk = j % C::kStagesK;
+            ROWS_T(12);
             wait_or_flag(bar(kBarKFull + sk), (j / C::kStagesK) & 1, p.status);
+            ROWS_T(8);
             if (j >= 2) wait_or_flag(bar(kBarSFree + s), ((j >> 1) - 1) & 1, p.status);
+            ROWS_T(9);
             if (lane == 0) {
                 tc_fence_after();
                 const uint64_t dK = make_smem_desc(base + C::kOffK + sk * kTileKV, 0, 1024);
@@ -328,8 +358,11 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         for (int j = 0; j < n_tiles; ++j) {
             const int sv = j % C::kStagesV;
             if (j + 1 < n_tiles) score(j + 1);  // runs while the element-wise warps work on tile j
+            ROWS_T(12);
             wait_or_flag(bar(kBarPFull), j & 1, p.status);
+            ROWS_T(10);
             wait_or_flag(bar(kBarVFull + sv), (j / C::kStagesV) & 1, p.status);
+            ROWS_T(11);
             if (lane == 0) {
                 tc_fence_after();
                 const uint64_t dV = make_smem_desc(base + C::kOffV + sv * kTileKV, kBoxKV, 1024);
@@ -344,9 +377,10 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             }
             __syncwarp();
         }
+        if (lane == 0) ROWS_FLUSH(8);
     } else {
         // ===================== element-wise warps =====================
-        // thread = (key of the tile = TMEM lane, half of the rows)
+        // thread = (key of the tile = TMEM lane, eight of the rows)
         const int quarter = warp & 3, part = warp >> 2;
         const int kr = quarter * 32 + lane;
         const int c0 = RPT * part;  // first row of this thread's columns
@@ -358,6 +392,7 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         // bit c: row c0 + c exists (fewer than NR rows: the padding rows take part with weights of zero)
         const uint32_t row_mask = p.rows - c0 >= RPT ? (1u << RPT) - 1u : (p.rows > c0 ? (1u << (p.rows - c0)) - 1u : 0u);
         const float4* const ref4 = reinterpret_cast<const float4*>(ref + c0);
+        ROWS_T0;
 
         for (int j = 0; j < n_tiles; ++j) {
             const int s = j & 1, sv = j % C::kStagesV;
@@ -377,7 +412,9 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 }
                 vis &= row_mask;
             }
+            ROWS_T(7);
             wait_or_flag(bar(kBarSFull + s), (j >> 1) & 1, p.status);
+            ROWS_T(0);
             tc_fence_after();
             uint32_t a[RPT], g[RPT];
             ld_cols(Sb + c0, a);
@@ -401,14 +438,17 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                     flag |= ((vis >> c) & 1u) && (!seen || x[c] > kRowsLazyThreshold);
                 }
             }
-            if (ew_barrier_or(flag)) {
+            ROWS_T(1);
+            const bool moved = ew_barrier_or<kEwThreads>(flag);
+            ROWS_T(2);
+            if (moved) {
                 // ---- some reference has to move: the tile's maximum of every row over its visible keys ----
                 float v[RPT];
 #pragma unroll
                 for (int c = 0; c < RPT; ++c) v[c] = ((vis >> c) & 1u) ? __uint_as_float(a[c]) * p.scale_log2e : -INFINITY;
                 const float m = warp_transpose_reduce<RPT, true>(v, lane);
                 if (lane < RPT) wmax[warp * RPT + lane] = m;
-                ew_barrier();
+                ew_barrier<kEwThreads>();
                 if (threadIdx.x < NR) {
                     const int row = threadIdx.x, pr = row / RPT, c = row % RPT;
                     const float tm = fmaxf(fmaxf(wmax[(4 * pr + 0) * RPT + c], wmax[(4 * pr + 1) * RPT + c]),
@@ -421,7 +461,7 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                     }
                     alpha[row] = al;
                 }
-                ew_barrier();
+                ew_barrier<kEwThreads>();
                 if (j > 0) {
                     // move the accumulated state to the new references (this thread's TMEM lane is a head dimension here)
                     wait_or_flag(bar(kBarPvDone), (j - 1) & 1, p.status);
@@ -454,6 +494,7 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 }
             }
 
+            ROWS_T(6);
             // ---- weights, row sums, bf16 parts and residuals ----
             uint32_t w4[4][RPT / 2];  // P1, P1 residual, P2, P2 residual: two rows per word
 #pragma unroll
@@ -474,7 +515,9 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 w4[3][c >> 1] = pack2(p2[0] - __low2float(b2), p2[1] - __high2float(b2));
             }
 
+            ROWS_T(3);
             if (j > 0) wait_or_flag(bar(kBarPvDone), (j - 1) & 1, p.status);  // the previous weight tile has been consumed
+            ROWS_T(4);
             // weight tile: [128 keys][4 NR columns] bf16 in 64-column blocks of 128 bytes per key, 128-byte swizzle
             // (chunk index XOR key mod 8); column which * NR + row
 #pragma unroll
@@ -501,7 +544,9 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             }
             fence_proxy_async_smem();
             mbar_arrive(bar(kBarPFull));
+            ROWS_T(5);
         }
+        if (threadIdx.x == 0) ROWS_FLUSH(0);
 
         // ---- row sums over the keys, then the epilogue: this thread's TMEM lane is head dimension kr ----
         wait_or_flag(bar(kBarFinal), 0, p.status);
@@ -515,7 +560,7 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 dsum[(warp * RPT + lane) * 2 + 1] = t2;
             }
         }
-        ew_barrier();
+        ew_barrier<kEwThreads>();
         float* const dtot = dsum + kEwWarps * RPT * 2;
         if (threadIdx.x < NR) {
             const int row = threadIdx.x, pr = row / RPT, c = row % RPT;
@@ -528,7 +573,7 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             dtot[2 * row] = t1;
             dtot[2 * row + 1] = t2;
         }
-        ew_barrier();
+        ew_barrier<kEwThreads>();
         {
             uint32_t u0[RPT], u1[RPT], w0[RPT], w1[RPT];
             ld_cols(lane_base + C::kColO + 0 * NR + c0, u0);
@@ -585,7 +630,7 @@ int launch_rows(const CUtensorMap& tmQ, const CUtensorMap& tmR, const CUtensorMa
             return PLX_ERR_CUDA;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    plx_decode_rows_kernel<NR><<<grid, kRowsThreads, RowsCfg<NR>::kSmemBytes, stream>>>(tmQ, tmR, tmK, tmV, rp);
+    plx_decode_rows_kernel<NR><<<grid, RowsCfg<NR>::kThreads, RowsCfg<NR>::kSmemBytes, stream>>>(tmQ, tmR, tmK, tmV, rp);
     return cudaGetLastError() == cudaSuccess ? PLX_OK : PLX_ERR_CUDA;
 }
 
@@ -682,6 +727,18 @@ int plx_decode_rows_fwd(const void* q, const void* r, const void* k_cache, const
                                           out_dtype, stream);
     return PLX_OK;
 }
+
+#if PLX_TRACE
+extern "C" int plx_rows_trace_read(long long* host, int n, int reset)
+{
+    if (cudaMemcpyFromSymbol(host, g_rows_trace, n * sizeof(long long)) != cudaSuccess) return PLX_ERR_CUDA;
+    if (reset) {
+        long long zeros[32] = {0};
+        if (cudaMemcpyToSymbol(g_rows_trace, zeros, sizeof zeros) != cudaSuccess) return PLX_ERR_CUDA;
+    }
+    return PLX_OK;
+}
+#endif
 
 extern "C" int parallax_decode_fwd_rows(const void* q, const void* r, const void* k_cache, const void* v_cache,
                                         const int32_t* seqlens, void* out, int B, int Hq, int Hkv, int D, int Lq,
