@@ -355,11 +355,11 @@ int parallax_decode_fwd_paged_fp8(const void* q, const void* r, const void* k_pa
  * query head are handled like Lq more query heads of its KV head (split-KV, fused merge and the
  * bandwidth-bound streaming of the decode kernel apply), so the call is HBM-bound where the
  * tensor-core multi-token kernel would compute a 128-row tile for a handful of rows.  That holds up
- * to eight rows per KV head (Lq * Hq / Hkv <= 8: above four rows several CTAs read the same K/V
- * through L2); larger steps are handed to parallax_prefill_fwd_ex (residual weights, its split
- * records in the same workspace), which is faster from there on at every batch size, so the call
- * accepts any Lq.  (Steps of 9..64 rows whose q, r or out is not 16-byte aligned stay on the decode
- * kernel; parallax_decode_fwd_args always does.)  Workspace as parallax_decode_fwd_ex for Hq * Lq
+ * to eight rows per KV head (Lq * Hq / Hkv <= 8, one CTA per KV head).  Nine to 32 rows at D = 128 run
+ * on the tensor-core kernel of parallax_decode_fwd_rows (keys on the accumulator lanes), larger steps
+ * and D = 64 on parallax_prefill_fwd_ex (residual weights); both keep their split records in the same
+ * workspace, so the call accepts any Lq.  (Steps of 9..64 rows whose q, r or out is not 16-byte
+ * aligned stay on the decode kernel; parallax_decode_fwd_args always does.)  Workspace as parallax_decode_fwd_ex for Hq * Lq
  * query heads (parallax_decode_workspace_bytes(B, Hq * Lq, D, max_splits)); everything else as there.
  */
 int parallax_decode_fwd_multi(const void* q, const void* r, const void* k_cache, const void* v_cache,
@@ -384,7 +384,8 @@ int parallax_decode_fwd_rows(const void* q, const void* r, const void* k_cache, 
                              int num_splits, int32_t* status, void* stream);
 
 /* parallax_decode_fwd_multi over the paged cache of parallax_decode_fwd_paged (q, r, out [B, Hq, Lq, D]);
- * the hand-over to the tensor-core kernel needs page_size to be a multiple of 64. */
+ * the hand-over to the keys-on-lanes kernel needs a page_size that divides 128 or is a multiple of it,
+ * the hand-over to the row-major tensor-core kernel a multiple of 64. */
 int parallax_decode_fwd_multi_paged(const void* q, const void* r, const void* k_pages, const void* v_pages,
                                     const int32_t* block_table, const int32_t* seqlens, void* out, int B,
                                     int Hq, int Hkv, int D, int Lq, int num_pages, int page_size,

@@ -1731,8 +1731,10 @@ int parallax_decode_fwd_fp8(const void* q, const void* r, const void* k_cache, c
 }
 
 // Which kernel takes a step of `rows` = (query heads per KV head) x (new tokens) rows per KV head.  Up to eight
-// rows one CTA of the decode kernel serves a KV head and is the faster route at every batch size.  Nine to sixteen
-// rows that split into two CTAs of at most eight (10 = 2 x 5, 12, 14, 16) stay on the decode kernel as well: measured
+// rows one CTA of the decode kernel serves a KV head and is the faster route at every batch size.  Nine to 32 rows at
+// D = 128 go to the keys-on-lanes tensor-core kernel (parallax_decode_fwd_multi decides that before it asks here).
+// For what that kernel does not serve (D = 64, other page sizes): nine to sixteen rows that split into two CTAs of at
+// most eight (10 = 2 x 5, 12, 14, 16) stay on the decode kernel, the rest goes to the row-major tensor-core kernel: measured
 // at 10 / 12 / 16 rows, 8 KV heads, decode kernel against the split-KV tensor-core kernel: 64 x 8192 keys 505 / 525 /
 // 533 us against 728 / 754 / 795; 12 x 8192 100 / 101 / 108 against 170 / 173 / 173; 8 x 8192 72 / 72 / 78 against
 // 103 / 103 / 95; 4 x 16384 72 / 72 / 79 against 93 / 93 / 103; 2 x 131072 291 / 298 / 332 against 322 / 376 / 366;

@@ -1,6 +1,7 @@
 """GPU parity of the multi-token decode step against the fp64 oracle of the multi-token causal forward.
 parallax_decode_fwd_multi runs up to eight rows per KV head on the decode kernel and hands larger steps to
-the tensor-core kernel; parallax_decode_fwd_args always stays on the decode kernel.  Every case runs through
+the tensor-core kernels (keys on the lanes up to 32 rows at D = 128, row-major above); parallax_decode_fwd_args
+always stays on the decode kernel.  Every case runs through
 both entries, so the decode kernel's per-head key counts are covered at every row count."""
 import numpy as np
 import pytest
