@@ -81,11 +81,12 @@ def test_rows_split_boundary_inside_the_new_tokens(plx, oracle):
         run_rows(plx, oracle, cfg, Lq, ns=(T + 127) // 128)
 
 
+@pytest.mark.parametrize("Lq", [8, 14])
 @pytest.mark.parametrize("kind", ["peaked", "growing"])
-def test_rows_reference_moves_late(plx, oracle, kind):
+def test_rows_reference_moves_late(plx, oracle, kind, Lq):
     """Scores that keep growing along the context (the reference exponent moves in many tiles, the accumulators are
-    rescaled in TMEM each time) and one dominant key late in the context."""
-    Lq, T = 8, 2048
+    rescaled in TMEM each time) and one dominant key late in the context; at 16 and 28 rows per KV head."""
+    T = 2048
     cfg = wl.DecodeConfig("rows " + kind, B=2, Hq=4, Hkv=2, D=128, T_max=T, seed=2500)
     x = wl.make_prefill_inputs(cfg, Lq, "cuda")
     if kind == "peaked":
