@@ -539,6 +539,9 @@ def run_ours(args, rank, world, local_rank):
         by_bytes = roofline.get("read_probe", {}).get("GBps_by_call_bytes")
         result["other_configs"] = {n: quick_config(n, sampler, read_peak, by_bytes) for n in sorted(wl.CONFIGS) if n != args.workload}
         result["other_workloads"] = {n: quick_tensor_workload(n, local_rank) for n in ("P2", "T1")}
+        for Lq in (4, 8):   # multi-token decode steps on the headline shape: 8 and 16 rows per KV head
+            result["other_workloads"][f"{args.workload}_new_tokens_{Lq}"] = quick_multi_token(args.workload, Lq, sampler, read_peak)
+            torch.cuda.empty_cache()
     if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.fp8_kv and Lq == 1:
         secs, nbytes, threads, desc = oracle_sample_time(cfg, x0, seqlens_host, args.cpu_seconds)
         result["cpu_baseline"] = {"value": round(nbytes / secs / 1e12, 8), "unit": UNIT, "cores": threads,
@@ -671,6 +674,35 @@ def quick_tensor_workload(name, local_rank=0):
     if name in wl.PREFILL_CONFIGS:   # the same workload with residual products only where rows see few keys
         res["p_precision"] = "bf16+residual"
         res["adaptive_p_precision"] = one("adaptive")
+    return res
+
+
+def quick_multi_token(name, Lq, sampler, read_peak=None, steps=20, warmup=5):
+    """Device-timed multi-token decode step (Lq new tokens per sequence through parallax_decode_fwd_multi, which
+    picks the kernel) on a decode configuration, for the default line: us per step, KV-read TB/s, tokens/s, kernel."""
+    from paper_2605_29157_b200 import binding as plx
+    cfg = wl.CONFIGS[name]
+    sets = [wl.make_prefill_inputs(wl.scaled(cfg, seed=cfg.seed + 17 * i), Lq, "cuda") for i in range(2)]
+    kv_bytes = cfg.kv_bytes(None)
+    ws = plx.alloc_workspace(cfg.B, cfg.Hq * Lq, cfg.D, plx.PLX_MAX_SPLITS, "cuda")
+    out = torch.empty(cfg.B, cfg.Hq, Lq, cfg.D, dtype=torch.bfloat16, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        x = sets[i % 2]
+        plx.parallax_decode_fwd_multi(x["q"], x["r"], x["k"], x["v"], None, out, cfg.scale, ws, 0, stream)
+    for i in range(warmup):
+        step(i)
+    t = BlockTimer(stream, sampler).run(step, steps)
+    assert plx.parallax_workspace_status(ws) == 0, "device-side wait timed out"
+    us = t["ms_per_step"] * 1e3
+    route = multi_token_route(cfg, Lq)
+    res = {"new_tokens_per_step": Lq, "rows_per_kv_head": cfg.G * Lq, "us_per_step": round(us, 2),
+           "kv_read_TBps": round(kv_bytes / us / 1e6, 4), "tokens_per_s": round(cfg.B * Lq / (us * 1e-6), 1),
+           "kernel": {"decode": "plx_decode_kernel", "rows": "plx_decode_rows_kernel", "row-major": "plx_prefill_kernel"}[route],
+           "clocks": t["clocks"], **timing_note(t)}
+    if read_peak:
+        res["frac_of_read_probe"] = round(kv_bytes / us / 1e3 / read_peak, 4)
     return res
 
 

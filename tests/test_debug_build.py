@@ -93,3 +93,37 @@ def test_a_page_id_outside_the_pool_is_reported_not_followed(dbg):
     dbg.parallax_decode_fwd_paged(x["q"], x["r"], kp, vp, good, None, out, cfg.scale, ws, 1)
     torch.cuda.synchronize()
     assert dbg.parallax_workspace_status(ws) == 0
+
+
+@pytest.mark.gpu
+def test_multi_token_step_through_the_checking_build(dbg, oracle):
+    """Twelve and 24 rows per KV head (the keys-on-lanes kernel) through the checking build: same results over a
+    contiguous and a paged cache; a page id outside the pool is reported through the status word, not followed."""
+    Lq = 6
+    for G in (2, 4):
+        cfg = wl.DecodeConfig("dbg-rows", B=3, Hq=2 * G, Hkv=2, D=128, T_max=900, ragged=(Lq, 900), seed=91 + G)
+        x = wl.make_prefill_inputs(cfg, Lq, "cuda")
+        bits = {n: wl.bf16_bits(x[n]) for n in ("q", "r", "k", "v")}
+        want, _ = oracle.prefill_bf16(bits["q"], bits["r"], bits["k"], bits["v"], x["seqlens_host"], cfg.scale)
+        out = torch.full((cfg.B, cfg.Hq, Lq, cfg.D), float("nan"), dtype=torch.float32, device="cuda")
+        ws = dbg.alloc_workspace(cfg.B, cfg.Hq * Lq, cfg.D, 8, "cuda")
+        dbg.parallax_decode_fwd_multi(x["q"], x["r"], x["k"], x["v"], x["seqlens"], out, cfg.scale, ws, 0)
+        torch.cuda.synchronize()
+        assert dbg.parallax_workspace_status(ws) == 0
+        assert_parity(out.cpu().numpy(), want, torch.float32, f"checking build, {G * Lq} rows")
+        kp, vp, table = wl.to_paged(x["k"], x["v"], 32, seed=4)
+        out.fill_(float("nan"))
+        dbg.parallax_decode_fwd_multi_paged(x["q"], x["r"], kp, vp, table, x["seqlens"], out, cfg.scale, ws, 3)
+        torch.cuda.synchronize()
+        assert dbg.parallax_workspace_status(ws) == 0
+        assert_parity(out.cpu().numpy(), want, torch.float32, f"checking build, paged, {G * Lq} rows")
+    bad = table.clone()
+    bad[0, 0] = kp.shape[0] + 17
+    dbg.parallax_decode_fwd_multi_paged(x["q"], x["r"], kp, vp, bad, x["seqlens"], out, cfg.scale, ws, 1)
+    torch.cuda.synchronize()
+    assert dbg.parallax_workspace_status(ws) == dbg.PLX_ERR_DEVICE_CHECK
+    assert torch.isfinite(out).all()
+    ws.zero_()
+    dbg.parallax_decode_fwd_multi_paged(x["q"], x["r"], kp, vp, table, x["seqlens"], out, cfg.scale, ws, 1)
+    torch.cuda.synchronize()
+    assert dbg.parallax_workspace_status(ws) == 0
