@@ -553,14 +553,14 @@ def run_ours(args, rank, world, local_rank):
 
 def multi_token_route(cfg, Lq, page_size=0):
     """Mirrors the library's routing of a multi-token step (only to name the kernel and count launches): up to
-    eight rows per KV head the decode kernel; nine to 32 rows at D = 128 the keys-on-lanes tensor-core kernel
+    eight rows per KV head the decode kernel; nine to 32 rows the keys-on-lanes tensor-core kernel
     ("rows"; paged caches when the page size divides 128 or is a multiple of it); otherwise nine to sixteen rows
     that split into two CTAs of at most eight stay on the decode kernel and everything else goes to the row-major
     tensor-core kernel."""
     rows = cfg.G * Lq
     if rows <= 8:
         return "decode"
-    if rows <= 32 and cfg.D == 128 and (not page_size or 128 % page_size == 0 or page_size % 128 == 0):
+    if rows <= 32 and cfg.D in (64, 128) and (not page_size or 128 % page_size == 0 or page_size % 128 == 0):
         return "rows"
     if rows <= 16:
         g = max(c for c in range(1, 9) if rows % c == 0)

@@ -355,9 +355,9 @@ int parallax_decode_fwd_paged_fp8(const void* q, const void* r, const void* k_pa
  * query head are handled like Lq more query heads of its KV head (split-KV, fused merge and the
  * bandwidth-bound streaming of the decode kernel apply), so the call is HBM-bound where the
  * tensor-core multi-token kernel would compute a 128-row tile for a handful of rows.  That holds up
- * to eight rows per KV head (Lq * Hq / Hkv <= 8, one CTA per KV head).  Nine to 32 rows at D = 128 run
+ * to eight rows per KV head (Lq * Hq / Hkv <= 8, one CTA per KV head).  Nine to 32 rows run
  * on the tensor-core kernel of parallax_decode_fwd_rows (keys on the accumulator lanes), larger steps
- * and D = 64 on parallax_prefill_fwd_ex (residual weights); both keep their split records in the same
+ * on parallax_prefill_fwd_ex (residual weights); both keep their split records in the same
  * workspace, so the call accepts any Lq.  (Steps of 9..64 rows whose q, r or out is not 16-byte
  * aligned stay on the decode kernel; parallax_decode_fwd_args always does.)  Workspace as parallax_decode_fwd_ex for Hq * Lq
  * query heads (parallax_decode_workspace_bytes(B, Hq * Lq, D, max_splits)); everything else as there.
@@ -370,7 +370,7 @@ int parallax_decode_fwd_multi(const void* q, const void* r, const void* k_cache,
 /*
  * The same step on the tensor-core kernel that keeps the KEYS on the accumulator lanes (Algorithm 1 with
  * S^T = K_c [Q; R]^T per 128-key tile and O^T += V_c^T P^T, so the tensor work follows the rows present):
- * up to 32 rows per KV head (Lq * Hq / Hkv <= 32), D = 128, bf16 caches, contiguous layout; q, r, k_cache,
+ * up to 32 rows per KV head (Lq * Hq / Hkv <= 32), D = 64 or 128, bf16 caches, contiguous layout; q, r, k_cache,
  * v_cache, out 16-byte aligned.  Split-KV like parallax_prefill_fwd_ex: `workspace` holds split records only
  * (parallax_prefill_workspace_bytes(B, Hq, D, Lq, max_splits) bytes, 16-byte aligned; NULL = one split),
  * num_splits 0 = planned (about one CTA per SM, at least four 128-key tiles per split), records merged by the

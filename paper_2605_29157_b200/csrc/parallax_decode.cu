@@ -1731,9 +1731,9 @@ int parallax_decode_fwd_fp8(const void* q, const void* r, const void* k_cache, c
 }
 
 // Which kernel takes a step of `rows` = (query heads per KV head) x (new tokens) rows per KV head.  Up to eight
-// rows one CTA of the decode kernel serves a KV head and is the faster route at every batch size.  Nine to 32 rows at
-// D = 128 go to the keys-on-lanes tensor-core kernel (parallax_decode_fwd_multi decides that before it asks here).
-// For what that kernel does not serve (D = 64, other page sizes): nine to sixteen rows that split into two CTAs of at
+// rows one CTA of the decode kernel serves a KV head and is the faster route at every batch size.  Nine to 32 rows
+// go to the keys-on-lanes tensor-core kernel (parallax_decode_fwd_multi decides that before it asks here).
+// For what that kernel does not serve (other page sizes, unaligned rows): nine to sixteen rows that split into two CTAs of at
 // most eight (10 = 2 x 5, 12, 14, 16) stay on the decode kernel, the rest goes to the row-major tensor-core kernel: measured
 // at 10 / 12 / 16 rows, 8 KV heads, decode kernel against the split-KV tensor-core kernel: 64 x 8192 keys 505 / 525 /
 // 533 us against 728 / 754 / 795; 12 x 8192 100 / 101 / 108 against 170 / 173 / 173; 8 x 8192 72 / 72 / 78 against
@@ -1774,12 +1774,14 @@ int parallax_decode_fwd_multi(const void* q, const void* r, const void* k_cache,
 {
     if (Lq <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || B <= 0) return PLX_ERR_BAD_SHAPE;
     if (workspace && !aligned(workspace, 16)) return PLX_ERR_ALIGNMENT;
-    // Nine to 32 rows per KV head at D = 128: the tensor-core kernel with the keys on the accumulator lanes, whose work
-    // follows the rows present.  Measured against the routes below (8 KV heads, 10 / 16 / 24 / 32 rows, us per step):
+    // Nine to 32 rows per KV head: the tensor-core kernel with the keys on the accumulator lanes, whose work
+    // follows the rows present.  Measured against the routes below (D = 128, 8 KV heads, 10 / 16 / 24 / 32 rows, us per step):
     // 64 x 8192 keys 342 / 352 / 412 / 462 against 474 / 506 / 722 / 766; 16 x 8192 94 / 92 / 107 / 108 against 146 / 154 /
     // 182 / 182; 8 x 8192 56 / 56 / 78 / 72 against 80 / 87 / 116 / 107; 2 x 131072 166 / 164 / 188 / 202 against 323 / 334 /
     // 339 / 339; 1 x 32768 36 / 37 / 44 / 45 against 52 / 59 / 57 / 58.  (Up to eight rows the decode kernel stays ahead
-    // or level at large batches: 64 x 8192, 2 / 4 / 8 rows: 298 / 300 / 314 against 324 / 329 / 340.)
+    // or level at large batches: 64 x 8192, 2 / 4 / 8 rows: 298 / 300 / 314 against 324 / 329 / 340.)  At D = 64, same
+    // shapes: 64 x 8192 278 / 286 / 370 / 381 against 305 / 309 / 570 / 570; 2 x 131072 131 / 132 / 168 / 169 against
+    // 153 / 152 / 267 / 267.
     if (static_cast<long long>(Hq / Hkv) * Lq > kMultiTokenDecodeRows && plx_decode_rows_supported(Hq, Hkv, D, Lq) &&
         aligned(q, 16) && aligned(r, 16) && aligned(out, 16) && aligned(k_cache, 16) && aligned(v_cache, 16)) {
         void* rec = nullptr;

@@ -2,7 +2,8 @@
 // times the query heads of a GQA group) on the tcgen05 tensor cores, with the KEYS on the TMEM lanes.
 //
 // The row-major multi-token kernel computes a 128-row tile whatever the number of rows, and the mma.sync decode
-// kernel is bound by its SM work from about ten rows on.  Here the work follows the rows present (NR = 16 or 32):
+// kernel is bound by its SM work from about ten rows on.  Here the work follows the rows present (NR = 16 or 32;
+// head dimension 128 or 64):
 //   S^T [128 keys x 2 NR]  = K_c [Q; R]^T                      one product per 128-key tile (Algorithm 1: S1, S2)
 //   O^T [D x 4 NR]        += V_c^T [P1 | P1 res | P2 | P2 res]^T  one product: A = the V tile read MN-major (head
 //                                                                dimension on M), B = the four weight tiles side by side
@@ -61,32 +62,33 @@ __device__ long long g_rows_trace[32];
 namespace {
 
 constexpr int BK = 128;  // keys per tile = TMEM lanes
-constexpr int HD = 128;  // head dimension
 constexpr int kMaxRows = 32;
 constexpr int kRowsPerThread = 8;              // rows per element-wise thread: NR / 8 threads share a key
-constexpr int kBoxKV = BK * 128;       // [128 keys x 64 columns] bf16 box: 16 KiB
-constexpr int kTileKV = 2 * kBoxKV;    // K or V tile
+constexpr int kBoxKV = BK * 128;       // [128 keys x 64 columns] bf16 box: 16 KiB (a K or V tile is HD / 64 of them)
 constexpr int kBlockP = BK * 128;      // [128 keys x 64 columns of the stacked weights] bf16: 16 KiB
-constexpr int kMaxStages = 3;
-enum : int { kBarQR = 0, kBarKFull = 1, kBarKFree = 4, kBarVFull = 7, kBarVFree = 10, kBarSFull = 13, kBarSFree = 15,
-             kBarPFull = 17, kBarPvDone = 18, kBarFinal = 19, kNumBars = 20 };
+constexpr int kMaxStages = 4;
+enum : int { kBarQR = 0, kBarKFull = 1, kBarKFree = 5, kBarVFull = 9, kBarVFree = 13, kBarSFull = 17, kBarSFree = 19,
+             kBarPFull = 21, kBarPvDone = 22, kBarFinal = 23, kNumBars = 24 };
 constexpr float kRowsLazyThreshold = 8.0f;       // log2 units
 constexpr float kLn2 = 0.6931471805599453f;
-constexpr int REC = 2 * HD + 4;
 
-// NR: rows of a KV head per CTA (the N extent of the weight tiles; fewer rows are padded)
-template <int NR>
+// NR: rows of a KV head per CTA (the N extent of the weight tiles; fewer rows are padded); HD: head dimension
+template <int NR, int HD>
 struct RowsCfg {
     static_assert(NR == 16 || NR == 32, "rows per KV head");
+    static_assert(HD == 64 || HD == 128, "head dimension");
+    static constexpr int kBoxes = HD / 64;                // 64-column boxes per row of Q, R, K, V
+    static constexpr int kTileKV = kBoxes * kBoxKV;       // K or V tile
+    static constexpr int REC = 2 * HD + 4;                // floats of a split record
     static constexpr int RPT = kRowsPerThread;
     static constexpr int kParts = NR / RPT;               // element-wise threads per key (2 or 4)
     static constexpr int kEwWarps = 4 * kParts;           // four warps cover the 128 keys (TMEM lanes) of a tile
     static constexpr int kEwThreads = kEwWarps * 32;
     static constexpr int kMmaWarp = kEwWarps, kTmaWarp = kEwWarps + 1;
     static constexpr int kThreads = (kEwWarps + 2) * 32;
-    static constexpr int kStagesK = NR == 16 ? 3 : 2, kStagesV = 3;
+    static constexpr int kStagesK = HD == 64 ? 4 : NR == 16 ? 3 : 2, kStagesV = HD == 64 ? 4 : 3;
     static constexpr int kBoxQR = 2 * NR * 128;           // [Q rows; R rows] x 64 columns: the N = 2 NR operand of the score product
-    static constexpr int kTileQR = 2 * kBoxQR;
+    static constexpr int kTileQR = kBoxes * kBoxQR;
     static constexpr int kPBlocks = 4 * NR / 64;          // 64-wide blocks of [P1 | P1 res | P2 | P2 res]
     static constexpr int kTileP = kPBlocks * kBlockP;
     static constexpr int kOffQR = 0;
@@ -180,13 +182,14 @@ __device__ __forceinline__ void store_value(void* out, size_t idx, float v, int 
 // complete a second phase before its waiter has seen the first: the S buffers alternate (a full / free pair per
 // buffer), the weight tiles are single (P full <-> P.V done hand over one tile at a time), the K and V rings
 // have a full / free pair per stage.
-template <int NR>
-__global__ void __launch_bounds__(RowsCfg<NR>::kThreads, 1)
+template <int NR, int HD>
+__global__ void __launch_bounds__(RowsCfg<NR, HD>::kThreads, 1)
 plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmR,
                        const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                        const RowsParams p)
 {
-    using C = RowsCfg<NR>;
+    using C = RowsCfg<NR, HD>;
+    constexpr int kTileKV = C::kTileKV, kBoxes = C::kBoxes, REC = C::REC;
     constexpr int RPT = C::RPT, kEwWarps = C::kEwWarps, kEwThreads = C::kEwThreads, kMmaWarp = C::kMmaWarp,
                   kTmaWarp = C::kTmaWarp, kRowsThreads = C::kThreads;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -262,7 +265,7 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             prefetch_tensormap(&tmV);
             mbar_expect_tx(bar(kBarQR), C::kTileQR);
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
+            for (int h = 0; h < kBoxes; ++h) {
                 tma_load_2d(base + C::kOffQR + h * C::kBoxQR, &tmQ, bar(kBarQR), 64 * h, static_cast<int>(row0));
                 tma_load_2d(base + C::kOffQR + h * C::kBoxQR + NR * 128, &tmR, bar(kBarQR), 64 * h, static_cast<int>(row0));
             }
@@ -278,14 +281,14 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                     const int krow = static_cast<int>(kv_row0) + key0;
                     mbar_expect_tx(bar(kBarKFull + sk), kTileKV);
 #pragma unroll
-                    for (int h = 0; h < 2; ++h)
+                    for (int h = 0; h < kBoxes; ++h)
                         tma_load_2d(base + C::kOffK + sk * kTileKV + h * kBoxKV, &tmK, bar(kBarKFull + sk), 64 * h, krow);
                     ROWS_T(18);
                     if (j >= C::kStagesV) wait_or_flag(bar(kBarVFree + sv), (j / C::kStagesV - 1) & 1, p.status);
                     ROWS_T(17);
                     mbar_expect_tx(bar(kBarVFull + sv), kTileKV);
 #pragma unroll
-                    for (int h = 0; h < 2; ++h)
+                    for (int h = 0; h < kBoxes; ++h)
                         tma_load_2d(base + C::kOffV + sv * kTileKV + h * kBoxKV, &tmV, bar(kBarVFull + sv), 64 * h, krow);
                 } else {
                     // Paged: the tile is fetched in boxes of page_box keys, each from its page.  Boxes that lie wholly
@@ -306,18 +309,18 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 #endif
                         rows_of[i] = (id * p.Hkv + hkv) * p.page_size + (key - pg * p.page_size);
                     }
-                    const uint32_t bytes = static_cast<uint32_t>(nbox) * pb * 128 * 2;
+                    const uint32_t bytes = static_cast<uint32_t>(nbox) * pb * 128 * kBoxes;
                     mbar_expect_tx(bar(kBarKFull + sk), bytes);
                     for (int i = 0; i < nbox; ++i)
 #pragma unroll
-                        for (int h = 0; h < 2; ++h)
+                        for (int h = 0; h < kBoxes; ++h)
                             tma_load_2d(base + C::kOffK + sk * kTileKV + h * kBoxKV + i * pb * 128, &tmK, bar(kBarKFull + sk),
                                         64 * h, rows_of[i]);
                     if (j >= C::kStagesV) wait_or_flag(bar(kBarVFree + sv), (j / C::kStagesV - 1) & 1, p.status);
                     mbar_expect_tx(bar(kBarVFull + sv), bytes);
                     for (int i = 0; i < nbox; ++i)
 #pragma unroll
-                        for (int h = 0; h < 2; ++h)
+                        for (int h = 0; h < kBoxes; ++h)
                             tma_load_2d(base + C::kOffV + sv * kTileKV + h * kBoxKV + i * pb * 128, &tmV, bar(kBarVFull + sv),
                                         64 * h, rows_of[i]);
                 }
@@ -328,7 +331,10 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     } else if (warp == kMmaWarp) {
         // ===================== score products and value products, one issuing thread =====================
         constexpr uint32_t idesc_s = make_idesc(BK, 2 * NR, 0, 0);   // K-major A (K tile), K-major B ([Q; R])
-        constexpr uint32_t idesc_pv = make_idesc(HD, 4 * NR, 1, 1);  // MN-major A (V tile: head dimension on M), MN-major B (weights)
+        // MN-major A (V tile: head dimension on M), MN-major B (weights).  M is 128 at either head dimension: at 64 the
+        // second 64-wide block of A is the first one again (block distance 0), so accumulator lanes 64-127 repeat
+        // lanes 0-63 and are ignored
+        constexpr uint32_t idesc_pv = make_idesc(128, 4 * NR, 1, 1);
         const uint64_t dQR = make_smem_desc(base + C::kOffQR, 0, 1024);
         const uint64_t dP = make_smem_desc(base + C::kOffP, kBlockP, 1024);
         wait_or_flag(bar(kBarQR), 0, p.status);
@@ -365,7 +371,7 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             ROWS_T(11);
             if (lane == 0) {
                 tc_fence_after();
-                const uint64_t dV = make_smem_desc(base + C::kOffV + sv * kTileKV, kBoxKV, 1024);
+                const uint64_t dV = make_smem_desc(base + C::kOffV + sv * kTileKV, HD == 128 ? kBoxKV : 0, 1024);
 #pragma unroll
                 for (int ks = 0; ks < BK / 16; ++ks) {
                     const uint64_t koff = static_cast<uint64_t>((ks * 2048) >> 4);
@@ -536,10 +542,8 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 if (key >= L) {
                     uint8_t* const vrow = smem + C::kOffV + sv * kTileKV + kr * 128;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        *reinterpret_cast<uint4*>(vrow + i * 16) = make_uint4(0u, 0u, 0u, 0u);
-                        *reinterpret_cast<uint4*>(vrow + kBoxKV + i * 16) = make_uint4(0u, 0u, 0u, 0u);
-                    }
+                    for (int i = 0; i < 8 * kBoxes; ++i)
+                        *reinterpret_cast<uint4*>(vrow + (i >> 3) * kBoxKV + (i & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
                 }
             }
             fence_proxy_async_smem();
@@ -584,7 +588,7 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 #pragma unroll
             for (int c = 0; c < RPT; ++c) {
                 const int row = c0 + c;
-                if (!((row_mask >> c) & 1u)) continue;
+                if (!((row_mask >> c) & 1u) || kr >= HD) continue;  // (head dimension 64: lanes 64-127 repeat lanes 0-63)
                 const float O1 = __uint_as_float(u0[c]) + __uint_as_float(u1[c]);
                 const float O2 = __uint_as_float(w0[c]) + __uint_as_float(w1[c]);
                 const float D1 = dtot[2 * row], D2 = dtot[2 * row + 1];
@@ -619,18 +623,18 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     }
 }
 
-template <int NR>
+template <int NR, int HD>
 int launch_rows(const CUtensorMap& tmQ, const CUtensorMap& tmR, const CUtensorMap& tmK, const CUtensorMap& tmV,
                 const RowsParams& rp, unsigned grid, int dev, cudaStream_t stream)
 {
     static bool configured[64] = {false};
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        if (cudaFuncSetAttribute(plx_decode_rows_kernel<NR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 RowsCfg<NR>::kSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(plx_decode_rows_kernel<NR, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 RowsCfg<NR, HD>::kSmemBytes) != cudaSuccess)
             return PLX_ERR_CUDA;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    plx_decode_rows_kernel<NR><<<grid, RowsCfg<NR>::kThreads, RowsCfg<NR>::kSmemBytes, stream>>>(tmQ, tmR, tmK, tmV, rp);
+    plx_decode_rows_kernel<NR, HD><<<grid, RowsCfg<NR, HD>::kThreads, RowsCfg<NR, HD>::kSmemBytes, stream>>>(tmQ, tmR, tmK, tmV, rp);
     return cudaGetLastError() == cudaSuccess ? PLX_OK : PLX_ERR_CUDA;
 }
 
@@ -641,7 +645,7 @@ int launch_rows(const CUtensorMap& tmQ, const CUtensorMap& tmR, const CUtensorMa
 // ---------------------------------------------------------------------------
 bool plx_decode_rows_supported(int Hq, int Hkv, int D, int Lq)
 {
-    return D == HD && Hkv > 0 && Hq % Hkv == 0 && Lq > 0 && static_cast<long long>(Hq / Hkv) * Lq <= kMaxRows;
+    return (D == 64 || D == 128) && Hkv > 0 && Hq % Hkv == 0 && Lq > 0 && static_cast<long long>(Hq / Hkv) * Lq <= kMaxRows;
 }
 
 // q, r, out [B, Hq, Lq, D]; `records` / `record_bytes`: room for split records (may be null: one split).
@@ -708,7 +712,7 @@ int plx_decode_rows_fwd(const void* q, const void* r, const void* k_cache, const
         } else {
             ns = num_splits < tiles_max ? num_splits : tiles_max;
         }
-        while (ns > 1 && static_cast<size_t>(q_rows) * ns * REC * sizeof(float) > record_bytes) --ns;
+        while (ns > 1 && static_cast<size_t>(q_rows) * ns * (2 * D + 4) * sizeof(float) > record_bytes) --ns;
     } else if (num_splits > 1) {
         return PLX_ERR_WORKSPACE;
     }
@@ -719,8 +723,12 @@ int plx_decode_rows_fwd(const void* q, const void* r, const void* k_cache, const
                   rows, ns, tps, scale * 1.4426950408889634f, out_dtype, block_table, page_size, max_pages, page_box, pool_rows};
     PlxNvtxRange nvtx_range("plx_decode_rows_fwd");
     const unsigned grid = static_cast<unsigned>(base_ctas * ns);
-    rc = nr == 16 ? launch_rows<16>(tmQ, tmR, tmK, tmV, rp, grid, dev, stream)
-                  : launch_rows<32>(tmQ, tmR, tmK, tmV, rp, grid, dev, stream);
+    if (D == 128)
+        rc = nr == 16 ? launch_rows<16, 128>(tmQ, tmR, tmK, tmV, rp, grid, dev, stream)
+                      : launch_rows<32, 128>(tmQ, tmR, tmK, tmV, rp, grid, dev, stream);
+    else
+        rc = nr == 16 ? launch_rows<16, 64>(tmQ, tmR, tmK, tmV, rp, grid, dev, stream)
+                      : launch_rows<32, 64>(tmQ, tmR, tmK, tmV, rp, grid, dev, stream);
     if (rc != PLX_OK) return rc;
     if (ns > 1)
         return plx_combine_after_producer(static_cast<const float*>(records), out, static_cast<int>(q_rows), D, ns,

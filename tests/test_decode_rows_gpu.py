@@ -106,6 +106,18 @@ def test_rows_reference_moves_late(plx, oracle, kind, Lq):
         assert_parity(out.cpu().numpy(), want, torch.float32, f"{kind} ns={ns}")
 
 
+@pytest.mark.parametrize("G,Lq", [(2, 8), (2, 16), (4, 3), (8, 4), (1, 1), (2, 5), (3, 7), (1, 32)])
+@pytest.mark.parametrize("T", [128, 200, 1000])
+def test_rows_head_dimension_64(plx, oracle, G, Lq, T):
+    """The same kernel at head dimension 64 (one 64-column box per row; the value product keeps M = 128 with its
+    second block repeating the first): single split, planned splits, ragged with NaN padding."""
+    cfg = wl.DecodeConfig("rows d64", B=2, Hq=2 * G, Hkv=2, D=64, T_max=T, seed=2800 + T + Lq)
+    run_rows(plx, oracle, cfg, Lq, ns=1)
+    if T == 1000:
+        run_rows(plx, oracle, cfg, Lq, ns=0, label="planned")
+        run_rows(plx, oracle, cfg, Lq, ns=3, seqlens=[max(1, Lq - 1), 777], label="ragged")
+
+
 def test_rows_rejects_what_it_does_not_serve(plx):
     q = torch.zeros(1, 4, 40, 128, dtype=torch.bfloat16, device="cuda")      # 80 rows per KV head
     k = torch.zeros(1, 2, 256, 128, dtype=torch.bfloat16, device="cuda")
@@ -113,9 +125,9 @@ def test_rows_rejects_what_it_does_not_serve(plx):
     with pytest.raises(plx.ParallaxError) as e:
         plx.parallax_decode_fwd_rows(q, q, k, k, None, out, 0.1)
     assert e.value.status == plx.PLX_ERR_UNSUPPORTED
-    q = torch.zeros(1, 4, 4, 64, dtype=torch.bfloat16, device="cuda")        # head dimension 64
-    k = torch.zeros(1, 2, 256, 64, dtype=torch.bfloat16, device="cuda")
-    out = torch.zeros(1, 4, 4, 64, dtype=torch.float32, device="cuda")
+    q = torch.zeros(1, 4, 4, 32, dtype=torch.bfloat16, device="cuda")        # head dimension 32
+    k = torch.zeros(1, 2, 256, 32, dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros(1, 4, 4, 32, dtype=torch.float32, device="cuda")
     with pytest.raises(plx.ParallaxError) as e:
         plx.parallax_decode_fwd_rows(q, q, k, k, None, out, 0.1)
     assert e.value.status == plx.PLX_ERR_UNSUPPORTED

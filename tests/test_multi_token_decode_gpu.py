@@ -1,6 +1,6 @@
 """GPU parity of the multi-token decode step against the fp64 oracle of the multi-token causal forward.
 parallax_decode_fwd_multi runs up to eight rows per KV head on the decode kernel and hands larger steps to
-the tensor-core kernels (keys on the lanes up to 32 rows at D = 128, row-major above); parallax_decode_fwd_args
+the tensor-core kernels (keys on the lanes up to 32 rows, row-major above); parallax_decode_fwd_args
 always stays on the decode kernel.  Every case runs through
 both entries, so the decode kernel's per-head key counts are covered at every row count."""
 import numpy as np
@@ -155,8 +155,8 @@ def test_multi_token_paged_cache(plx, oracle, page_size, Lq, T, ns):
 @pytest.mark.parametrize("D", [64, 128])
 @pytest.mark.parametrize("G,Lq", [(2, 5), (2, 6), (2, 8), (4, 4), (2, 7)])
 def test_ten_to_sixteen_rows(plx, oracle, D, G, Lq):
-    """10 / 12 / 14 / 16 rows per KV head: at D = 64 two CTAs of the decode kernel (five to eight rows each), at
-    D = 128 the keys-on-lanes tensor-core kernel (the options-struct entry stays on the decode kernel either way).
+    """10 / 12 / 14 / 16 rows per KV head: the keys-on-lanes tensor-core kernel through the multi-token entry, two
+    CTAs of the decode kernel (five to eight rows each) through the options-struct entry, at both head dimensions.
     Ragged contexts, NaN padding, planned splits."""
     B, Hkv = 16, 8
     cfg = wl.DecodeConfig("ten to sixteen rows", B=B, Hq=Hkv * G, Hkv=Hkv, D=D, T_max=700, seed=1700 + G * Lq)
