@@ -84,8 +84,8 @@ struct RowsCfg {
     static constexpr int kParts = NR / RPT;               // element-wise threads per key (2 or 4)
     static constexpr int kEwWarps = 4 * kParts;           // four warps cover the 128 keys (TMEM lanes) of a tile
     static constexpr int kEwThreads = kEwWarps * 32;
-    static constexpr int kMmaWarp = kEwWarps, kTmaWarp = kEwWarps + 1;
-    static constexpr int kThreads = (kEwWarps + 2) * 32;
+    static constexpr int kMmaWarp = kEwWarps, kPvWarp = kEwWarps + 1, kTmaWarp = kEwWarps + 2;
+    static constexpr int kThreads = (kEwWarps + 3) * 32;
     static constexpr int kStagesK = HD == 64 ? 4 : NR == 16 ? 3 : 2, kStagesV = HD == 64 ? 4 : 3;
     static constexpr int kBoxQR = 2 * NR * 128;           // [Q rows; R rows] x 64 columns: the N = 2 NR operand of the score product
     static constexpr int kTileQR = kBoxes * kBoxQR;
@@ -191,7 +191,7 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     using C = RowsCfg<NR, HD>;
     constexpr int kTileKV = C::kTileKV, kBoxes = C::kBoxes, REC = C::REC;
     constexpr int RPT = C::RPT, kEwWarps = C::kEwWarps, kEwThreads = C::kEwThreads, kMmaWarp = C::kMmaWarp,
-                  kTmaWarp = C::kTmaWarp, kRowsThreads = C::kThreads;
+                  kPvWarp = C::kPvWarp, kTmaWarp = C::kTmaWarp, kRowsThreads = C::kThreads;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t base = smem_u32(smem_raw);
     uint8_t* const smem = smem_raw;
@@ -328,8 +328,13 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             ROWS_FLUSH(16);
         }
         __syncwarp();
-    } else if (warp == kMmaWarp) {
-        // ===================== score products and value products, one issuing thread =====================
+    } else if (warp == kMmaWarp || warp == kPvWarp) {
+        // ===================== score products and value products =====================
+        // One issuing thread each.  At head dimension 64, where the element-wise and tensor work bound the step, the
+        // two run in warps of their own, so that the waits of one (K, the S buffer / the weights, V) do not delay the
+        // other: 13 % faster at sixteen rows.  At 128 the step is bound by HBM, a single issuer alternating between
+        // them measured level or a little better (2 x 131072 keys: 166 against 174 us), and the second warp idles.
+        constexpr bool kTwoIssuers = (HD == 64);
         constexpr uint32_t idesc_s = make_idesc(BK, 2 * NR, 0, 0);   // K-major A (K tile), K-major B ([Q; R])
         // MN-major A (V tile: head dimension on M), MN-major B (weights).  M is 128 at either head dimension: at 64 the
         // second 64-wide block of A is the first one again (block distance 0), so accumulator lanes 64-127 repeat
@@ -337,9 +342,8 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         constexpr uint32_t idesc_pv = make_idesc(128, 4 * NR, 1, 1);
         const uint64_t dQR = make_smem_desc(base + C::kOffQR, 0, 1024);
         const uint64_t dP = make_smem_desc(base + C::kOffP, kBlockP, 1024);
-        wait_or_flag(bar(kBarQR), 0, p.status);
         ROWS_T0;
-        auto score = [&](int j) {
+        auto score = [&](int j) {  // runs at most two tiles ahead of the element-wise warps (two S buffers)
             const int s = j & 1, sk = j % C::kStagesK;
             ROWS_T(12);
             wait_or_flag(bar(kBarKFull + sk), (j / C::kStagesK) & 1, p.status);
@@ -360,10 +364,8 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             }
             __syncwarp();
         };
-        score(0);
-        for (int j = 0; j < n_tiles; ++j) {
+        auto value = [&](int j) {
             const int sv = j % C::kStagesV;
-            if (j + 1 < n_tiles) score(j + 1);  // runs while the element-wise warps work on tile j
             ROWS_T(12);
             wait_or_flag(bar(kBarPFull), j & 1, p.status);
             ROWS_T(10);
@@ -382,8 +384,22 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 if (j == n_tiles - 1) tc_commit(bar(kBarFinal));
             }
             __syncwarp();
+        };
+        if (warp == kMmaWarp) {
+            wait_or_flag(bar(kBarQR), 0, p.status);
+            if constexpr (kTwoIssuers) {
+                for (int j = 0; j < n_tiles; ++j) score(j);
+            } else {
+                score(0);
+                for (int j = 0; j < n_tiles; ++j) {
+                    if (j + 1 < n_tiles) score(j + 1);  // runs while the element-wise warps work on tile j
+                    value(j);
+                }
+            }
+            if (lane == 0) ROWS_FLUSH(8);
+        } else if constexpr (kTwoIssuers) {
+            for (int j = 0; j < n_tiles; ++j) value(j);
         }
-        if (lane == 0) ROWS_FLUSH(8);
     } else {
         // ===================== element-wise warps =====================
         // thread = (key of the tile = TMEM lane, eight of the rows)
