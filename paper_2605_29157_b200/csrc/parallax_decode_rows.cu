@@ -446,18 +446,37 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             mbar_arrive(bar(kBarSFree + s));  // the score buffer is in registers
 
             // exponents against the references as they stand; does any visible score need a reference to move?
+            // `plain`: every row of this thread exists and sees every key of the tile (warp-uniform): packed
+            // arithmetic, no selects; a row without a reference yet gives x = +inf and raises the flag by itself
+            const bool plain = !need_mask && row_mask == (1u << RPT) - 1u;
             float x[RPT];
             bool flag = false;
+            if (plain) {
+                const uint64_t sc2 = pack_f2(p.scale_log2e, p.scale_log2e);
+                float mx = -INFINITY;
 #pragma unroll
-            for (int c4 = 0; c4 < RPT / 4; ++c4) {
-                const float4 r4 = ref4[c4];
-                const float rf[4] = {r4.x, r4.y, r4.z, r4.w};
+                for (int c4 = 0; c4 < RPT / 4; ++c4) {
+                    const float4 r4 = ref4[c4];
+                    const int c = 4 * c4;
+                    unpack_f2(fma2(pack_f2(__uint_as_float(a[c]), __uint_as_float(a[c + 1])), sc2, pack_f2(-r4.x, -r4.y)), x[c], x[c + 1]);
+                    unpack_f2(fma2(pack_f2(__uint_as_float(a[c + 2]), __uint_as_float(a[c + 3])), sc2, pack_f2(-r4.z, -r4.w)), x[c + 2],
+                              x[c + 3]);
+                    mx = max3(mx, x[c], x[c + 1]);
+                    mx = max3(mx, x[c + 2], x[c + 3]);
+                }
+                flag = mx > kRowsLazyThreshold;
+            } else {
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int c = 4 * c4 + e;
-                    const bool seen = rf[e] > -INFINITY;
-                    x[c] = fmaf(__uint_as_float(a[c]), p.scale_log2e, -(seen ? rf[e] : 0.0f));
-                    flag |= ((vis >> c) & 1u) && (!seen || x[c] > kRowsLazyThreshold);
+                for (int c4 = 0; c4 < RPT / 4; ++c4) {
+                    const float4 r4 = ref4[c4];
+                    const float rf[4] = {r4.x, r4.y, r4.z, r4.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int c = 4 * c4 + e;
+                        const bool seen = rf[e] > -INFINITY;
+                        x[c] = fmaf(__uint_as_float(a[c]), p.scale_log2e, -(seen ? rf[e] : 0.0f));
+                        flag |= ((vis >> c) & 1u) && (!seen || x[c] > kRowsLazyThreshold);
+                    }
                 }
             }
             ROWS_T(1);
@@ -519,22 +538,44 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             ROWS_T(6);
             // ---- weights, row sums, bf16 parts and residuals ----
             uint32_t w4[4][RPT / 2];  // P1, P1 residual, P2, P2 residual: two rows per word
+            if (plain) {
+                const uint64_t neg1 = pack_f2(-1.0f, -1.0f);
 #pragma unroll
-            for (int c = 0; c < RPT; c += 2) {
-                float p1[2], p2[2];
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const bool ok = (vis >> (c + e)) & 1u;
-                    p1[e] = ok ? ex2(x[c + e]) : 0.0f;
-                    p2[e] = ok ? p1[e] * __uint_as_float(g[c + e]) : 0.0f;
-                    d1[c + e] += p1[e];
-                    d2[c + e] += p2[e];
+                for (int c = 0; c < RPT; c += 2) {
+                    const uint64_t P1 = pack_f2(ex2(x[c]), ex2(x[c + 1]));
+                    const uint64_t P2 = mul2(P1, pack_f2(__uint_as_float(g[c]), __uint_as_float(g[c + 1])));
+                    unpack_f2(add2(pack_f2(d1[c], d1[c + 1]), P1), d1[c], d1[c + 1]);
+                    unpack_f2(add2(pack_f2(d2[c], d2[c + 1]), P2), d2[c], d2[c + 1]);
+                    float lo, hi;
+                    unpack_f2(P1, lo, hi);
+                    const uint32_t b1 = pack2(lo, hi);
+                    unpack_f2(P2, lo, hi);
+                    const uint32_t b2 = pack2(lo, hi);
+                    w4[0][c >> 1] = b1;
+                    w4[2][c >> 1] = b2;
+                    unpack_f2(fma2(bf16x2_to_f2(b1), neg1, P1), lo, hi);  // what the bf16 rounding left over
+                    w4[1][c >> 1] = pack2(lo, hi);
+                    unpack_f2(fma2(bf16x2_to_f2(b2), neg1, P2), lo, hi);
+                    w4[3][c >> 1] = pack2(lo, hi);
                 }
-                const __nv_bfloat162 b1 = __floats2bfloat162_rn(p1[0], p1[1]), b2 = __floats2bfloat162_rn(p2[0], p2[1]);
-                w4[0][c >> 1] = *reinterpret_cast<const uint32_t*>(&b1);
-                w4[2][c >> 1] = *reinterpret_cast<const uint32_t*>(&b2);
-                w4[1][c >> 1] = pack2(p1[0] - __low2float(b1), p1[1] - __high2float(b1));
-                w4[3][c >> 1] = pack2(p2[0] - __low2float(b2), p2[1] - __high2float(b2));
+            } else {
+#pragma unroll
+                for (int c = 0; c < RPT; c += 2) {
+                    float p1[2], p2[2];
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const bool ok = (vis >> (c + e)) & 1u;
+                        p1[e] = ok ? ex2(x[c + e]) : 0.0f;
+                        p2[e] = ok ? p1[e] * __uint_as_float(g[c + e]) : 0.0f;
+                        d1[c + e] += p1[e];
+                        d2[c + e] += p2[e];
+                    }
+                    const __nv_bfloat162 b1 = __floats2bfloat162_rn(p1[0], p1[1]), b2 = __floats2bfloat162_rn(p2[0], p2[1]);
+                    w4[0][c >> 1] = *reinterpret_cast<const uint32_t*>(&b1);
+                    w4[2][c >> 1] = *reinterpret_cast<const uint32_t*>(&b2);
+                    w4[1][c >> 1] = pack2(p1[0] - __low2float(b1), p1[1] - __high2float(b1));
+                    w4[3][c >> 1] = pack2(p2[0] - __low2float(b2), p2[1] - __high2float(b2));
+                }
             }
 
             ROWS_T(3);
