@@ -1776,12 +1776,11 @@ int parallax_decode_fwd_multi(const void* q, const void* r, const void* k_cache,
     if (workspace && !aligned(workspace, 16)) return PLX_ERR_ALIGNMENT;
     // Nine to 32 rows per KV head: the tensor-core kernel with the keys on the accumulator lanes, whose work
     // follows the rows present.  Measured against the routes below (D = 128, 8 KV heads, 10 / 16 / 24 / 32 rows, us per step):
-    // 64 x 8192 keys 342 / 352 / 412 / 462 against 474 / 506 / 722 / 766; 16 x 8192 94 / 92 / 107 / 108 against 146 / 154 /
-    // 182 / 182; 8 x 8192 56 / 56 / 78 / 72 against 80 / 87 / 116 / 107; 2 x 131072 166 / 164 / 188 / 202 against 323 / 334 /
-    // 339 / 339; 1 x 32768 36 / 37 / 44 / 45 against 52 / 59 / 57 / 58.  (Up to eight rows the decode kernel stays ahead
+    // 64 x 8192 keys 342 / 350 / 375 / 388 against 474 / 506 / 722 / 766; 16 x 8192 90 / 87 / 91 / 91 against 146 / 154 /
+    // 182 / 182; 8 x 8192 53 / 53 / 57 / 58 against 80 / 87 / 116 / 107; 2 x 131072 167 / 169 / 172 / 172 against 323 / 334 /
+    // 339 / 339; 1 x 32768 37 / 37 / 39 / 39 against 52 / 59 / 57 / 58.  (Up to eight rows the decode kernel stays ahead
     // or level at large batches: 64 x 8192, 2 / 4 / 8 rows: 298 / 300 / 314 against 324 / 329 / 340.)  At D = 64, same
-    // shapes: 64 x 8192 278 / 286 / 370 / 381 against 305 / 309 / 570 / 570; 2 x 131072 131 / 132 / 168 / 169 against
-    // 153 / 152 / 267 / 267.
+    // shapes, 16 / 32 rows: 64 x 8192 222 / 308 against 309 / 570; 2 x 131072 98 / 132 against 152 / 267.
     if (static_cast<long long>(Hq / Hkv) * Lq > kMultiTokenDecodeRows && plx_decode_rows_supported(Hq, Hkv, D, Lq) &&
         aligned(q, 16) && aligned(r, 16) && aligned(out, 16) && aligned(k_cache, 16) && aligned(v_cache, 16)) {
         void* rec = nullptr;
