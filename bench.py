@@ -539,8 +539,9 @@ def run_ours(args, rank, world, local_rank):
         by_bytes = roofline.get("read_probe", {}).get("GBps_by_call_bytes")
         result["other_configs"] = {n: quick_config(n, sampler, read_peak, by_bytes) for n in sorted(wl.CONFIGS) if n != args.workload}
         result["other_workloads"] = {n: quick_tensor_workload(n, local_rank) for n in ("P2", "T1")}
-        for Lq in (4, 8):   # multi-token decode steps on the headline shape: 8 and 16 rows per KV head
-            result["other_workloads"][f"{args.workload}_new_tokens_{Lq}"] = quick_multi_token(args.workload, Lq, sampler, read_peak)
+        for new_tokens in (4, 8):   # multi-token decode steps on the headline shape: 8 and 16 rows per KV head
+            result["other_workloads"][f"{args.workload}_new_tokens_{new_tokens}"] = quick_multi_token(args.workload, new_tokens,
+                                                                                                   sampler, read_peak)
             torch.cuda.empty_cache()
     if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.fp8_kv and Lq == 1:
         secs, nbytes, threads, desc = oracle_sample_time(cfg, x0, seqlens_host, args.cpu_seconds)

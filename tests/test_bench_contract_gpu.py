@@ -44,6 +44,17 @@ def test_decode_line_has_the_contract_keys(cuda_device):
     assert abs(d["value"] - kv_bytes / (d["ms_per_step"] * 1e-3) / 1e12) < 0.02 * d["value"]
 
 
+def test_default_line_has_every_section(cuda_device):
+    """The default invocation's shape (short steps, short CPU sample): the other decode configurations, the tensor-core
+    workloads, the multi-token steps and the CPU baseline are all there."""
+    d = _line("--workload", "C2", "--steps", "5", "--warmup", "3", "--cpu-seconds", "1")
+    assert set(d["other_configs"]) == {"C1", "C3", "C4", "C5", "C6"}
+    ow = d["other_workloads"]
+    assert {"P2", "T1", "C2_new_tokens_4", "C2_new_tokens_8"} <= set(ow)
+    assert ow["C2_new_tokens_8"]["kernel"] == "plx_decode_rows_kernel" and ow["C2_new_tokens_4"]["kernel"] == "plx_decode_kernel"
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["sustained"]["value"] > 0
+
+
 def test_sharded_line_on_one_rank(cuda_device):
     d = _line("--gpus", "1", "--shard-keys", "--workload", "C2", "--steps", "5")
     assert d["scaling"] == "strong" and d["n_gpus"] == 1 and d["e2e"]["value"] > 0
