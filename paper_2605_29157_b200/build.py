@@ -22,7 +22,7 @@ SOURCES = [PKG / "csrc" / "parallax_decode.cu", PKG / "csrc" / "parallax_prefill
            PKG / "csrc" / "parallax_prepare.cu", PKG / "csrc" / "parallax_backward.cu",
            PKG / "csrc" / "parallax_probe.cu", PKG / "csrc" / "parallax_decode_rows.cu"]
 HEADERS = [ROOT / "include" / "parallax.h", ROOT / "include" / "parallax_test_hooks.h",
-           PKG / "csrc" / "plx_common.cuh", PKG / "csrc" / "plx_tcgen05.cuh"]
+           PKG / "csrc" / "plx_common.cuh", PKG / "csrc" / "plx_tcgen05.cuh", PKG / "csrc" / "plx_internal.h"]
 LIB = PKG / "libparallax.so"
 LIB_DEBUG = PKG / "libparallax_debug.so"
 

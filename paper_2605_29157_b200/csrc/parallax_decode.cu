@@ -32,15 +32,7 @@
 
 #include "parallax.h"
 #include "plx_common.cuh"
-
-// Defined in parallax_decode_rows.cu: multi-token decode steps of up to 32 rows per KV head on the tensor cores with
-// the keys on the accumulator lanes.
-bool plx_decode_rows_supported(int Hq, int Hkv, int D, int Lq);
-bool plx_decode_rows_page_size_ok(int page_size);
-int plx_decode_rows_fwd(const void* q, const void* r, const void* k_cache, const void* v_cache, const int32_t* seqlens,
-                        void* out, int B, int Hq, int Hkv, int D, int Lq, int T_max, float scale, int out_dtype,
-                        void* records, size_t record_bytes, int num_splits, int32_t* status, cudaStream_t stream,
-                        const int32_t* block_table, int page_size, int max_pages, long long pool_rows);
+#include "plx_internal.h"
 
 namespace {
 

@@ -24,11 +24,8 @@
 
 #include "parallax.h"
 #include "plx_common.cuh"
+#include "plx_internal.h"
 #include "plx_tcgen05.cuh"
-
-// Defined in parallax_decode.cu: the split merge launched as a programmatic dependent of the kernel before it.
-int plx_combine_after_producer(const float* partials, void* out, int rows, int D, int num_splits, int out_dtype,
-                               cudaStream_t stream);
 
 #ifndef PLX_DEBUG_CHECKS
 #define PLX_DEBUG_CHECKS 0  // 1: page ids are verified against the pool before they are followed
