@@ -413,7 +413,13 @@ def run_ours(args, rank, world, local_rank):
 
     def step(i, st=None):
         x, st = sets[i % nsets], st or stream
-        if Lq > 1:
+        if Lq > 1 and args.fp8_kv:      # several tokens over an e4m3 cache: the options-struct entry (decode kernel)
+            plx.parallax_decode_fwd_args(x["q"], x["r"], x["k8"], x["v8"], x["seqlens"], out, cfg.scale, k_scale=x["ks"],
+                                         v_scale=x["vs"], workspace=ws, num_splits=args.splits, stream=st)
+        elif Lq > 1 and args.page_size:
+            plx.parallax_decode_fwd_multi_paged(x["q"], x["r"], x["kp"], x["vp"], x["table"], x["seqlens"], out, cfg.scale,
+                                                ws, args.splits, st)
+        elif Lq > 1:
             plx.parallax_decode_fwd_multi(x["q"], x["r"], x["k"], x["v"], x["seqlens"], out, cfg.scale, ws, args.splits, st)
         elif args.page_size:
             plx.parallax_decode_fwd_paged(x["q"], x["r"], x["kp"], x["vp"], x["table"], x["seqlens"], out, cfg.scale,
