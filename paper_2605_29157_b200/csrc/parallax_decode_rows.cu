@@ -266,16 +266,16 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 tma_load_2d(base + C::kOffQR + h * C::kBoxQR, &tmQ, bar(kBarQR), 64 * h, static_cast<int>(row0));
                 tma_load_2d(base + C::kOffQR + h * C::kBoxQR + NR * 128, &tmR, bar(kBarQR), 64 * h, static_cast<int>(row0));
             }
-            const int32_t* const table = p.block_table ? p.block_table + static_cast<size_t>(b) * p.max_pages : nullptr;
-            ROWS_T0;
-            for (int j = 0; j < n_tiles; ++j) {
-                const int sk = j % C::kStagesK, sv = j % C::kStagesV;
-                const int key0 = (jt0 + j) * BK;
-                ROWS_T(18);
-                if (j >= C::kStagesK) wait_or_flag(bar(kBarKFree + sk), (j / C::kStagesK - 1) & 1, p.status);
-                ROWS_T(16);
-                if (!table) {
-                    const int krow = static_cast<int>(kv_row0) + key0;
+        }
+        if (!p.block_table) {
+            if (lane == 0) {
+                ROWS_T0;
+                for (int j = 0; j < n_tiles; ++j) {
+                    const int sk = j % C::kStagesK, sv = j % C::kStagesV;
+                    const int krow = static_cast<int>(kv_row0) + (jt0 + j) * BK;
+                    ROWS_T(18);
+                    if (j >= C::kStagesK) wait_or_flag(bar(kBarKFree + sk), (j / C::kStagesK - 1) & 1, p.status);
+                    ROWS_T(16);
                     mbar_expect_tx(bar(kBarKFull + sk), kTileKV);
 #pragma unroll
                     for (int h = 0; h < kBoxes; ++h)
@@ -287,42 +287,45 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 #pragma unroll
                     for (int h = 0; h < kBoxes; ++h)
                         tma_load_2d(base + C::kOffV + sv * kTileKV + h * kBoxKV, &tmV, bar(kBarVFull + sv), 64 * h, krow);
-                } else {
-                    // Paged: the tile is fetched in boxes of page_box keys, each from its page.  Boxes that lie wholly
-                    // past the context are not fetched (their pages need not exist): those rows of the tile keep what
-                    // an earlier tile left there, their scores are masked and their V rows are cleared before use.
-                    const int pb = p.page_box;
-                    const int nbox = min(BK / pb, (L - key0 + pb - 1) / pb);
-                    int rows_of[BK / 16];
-                    for (int i = 0; i < nbox; ++i) {
-                        const int key = key0 + i * pb;
-                        const int pg = key / p.page_size;
-                        int id = __ldg(table + pg);
-#if PLX_DEBUG_CHECKS
-                        if (id < 0 || (static_cast<long long>(id) * p.Hkv + hkv + 1) * p.page_size > p.pool_rows) {
-                            if (p.status) atomicExch(p.status, PLX_ERR_DEVICE_CHECK);  // a page id outside the pool: not followed
-                            id = 0;
-                        }
-#endif
-                        rows_of[i] = (id * p.Hkv + hkv) * p.page_size + (key - pg * p.page_size);
-                    }
-                    const uint32_t bytes = static_cast<uint32_t>(nbox) * pb * 128 * kBoxes;
-                    mbar_expect_tx(bar(kBarKFull + sk), bytes);
-                    for (int i = 0; i < nbox; ++i)
-#pragma unroll
-                        for (int h = 0; h < kBoxes; ++h)
-                            tma_load_2d(base + C::kOffK + sk * kTileKV + h * kBoxKV + i * pb * 128, &tmK, bar(kBarKFull + sk),
-                                        64 * h, rows_of[i]);
-                    if (j >= C::kStagesV) wait_or_flag(bar(kBarVFree + sv), (j / C::kStagesV - 1) & 1, p.status);
-                    mbar_expect_tx(bar(kBarVFull + sv), bytes);
-                    for (int i = 0; i < nbox; ++i)
-#pragma unroll
-                        for (int h = 0; h < kBoxes; ++h)
-                            tma_load_2d(base + C::kOffV + sv * kTileKV + h * kBoxKV + i * pb * 128, &tmV, bar(kBarVFull + sv),
-                                        64 * h, rows_of[i]);
                 }
+                ROWS_FLUSH(16);
             }
-            ROWS_FLUSH(16);
+        } else {
+            // Paged: the tile is fetched in boxes of page_box keys, each from its page, one (box, 64-column half) per
+            // lane of this warp (a page size of 16 means sixteen copies per tile and tensor).  Boxes that lie wholly
+            // past the context are not fetched (their pages need not exist): those rows of the tile keep what an
+            // earlier tile left there, their scores are masked and their V rows are cleared before use.
+            const int32_t* const table = p.block_table + static_cast<size_t>(b) * p.max_pages;
+            const int pb = p.page_box;
+            const int my_box = lane / kBoxes, my_half = lane % kBoxes;
+            for (int j = 0; j < n_tiles; ++j) {
+                const int sk = j % C::kStagesK, sv = j % C::kStagesV;
+                const int key0 = (jt0 + j) * BK;
+                const int nbox = min(BK / pb, (L - key0 + pb - 1) / pb);
+                const uint32_t bytes = static_cast<uint32_t>(nbox) * pb * 128 * kBoxes;
+                int row = 0;
+                if (my_box < nbox) {
+                    const int key = key0 + my_box * pb;
+                    const int pg = key / p.page_size;
+                    int id = __ldg(table + pg);
+#if PLX_DEBUG_CHECKS
+                    if (id < 0 || (static_cast<long long>(id) * p.Hkv + hkv + 1) * p.page_size > p.pool_rows) {
+                        if (p.status) atomicExch(p.status, PLX_ERR_DEVICE_CHECK);  // a page id outside the pool: not followed
+                        id = 0;
+                    }
+#endif
+                    row = (id * p.Hkv + hkv) * p.page_size + (key - pg * p.page_size);
+                }
+                const uint32_t off = static_cast<uint32_t>(my_half * kBoxKV + my_box * pb * 128);
+                if (j >= C::kStagesK) wait_or_flag(bar(kBarKFree + sk), (j / C::kStagesK - 1) & 1, p.status);
+                if (lane == 0) mbar_expect_tx(bar(kBarKFull + sk), bytes);
+                __syncwarp();
+                if (my_box < nbox) tma_load_2d(base + C::kOffK + sk * kTileKV + off, &tmK, bar(kBarKFull + sk), 64 * my_half, row);
+                if (j >= C::kStagesV) wait_or_flag(bar(kBarVFree + sv), (j / C::kStagesV - 1) & 1, p.status);
+                if (lane == 0) mbar_expect_tx(bar(kBarVFull + sv), bytes);
+                __syncwarp();
+                if (my_box < nbox) tma_load_2d(base + C::kOffV + sv * kTileKV + off, &tmV, bar(kBarVFull + sv), 64 * my_half, row);
+            }
         }
         __syncwarp();
     } else if (warp == kMmaWarp || warp == kPvWarp) {
