@@ -45,6 +45,14 @@ __device__ long long g_rows_trace[32];
         tr_acc[(i) & 7] += tr_now - tr_t;   \
         tr_t = tr_now;                      \
     } while (0)
+#define ROWS_STAMP(i)                                                              \
+    do {                                                                           \
+        if (blockIdx.x == 0 && threadIdx.x == 0) {                                 \
+            unsigned long long tr_g;                                               \
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tr_g));               \
+            g_rows_trace[24 + (i)] = static_cast<long long>(tr_g);                 \
+        }                                                                          \
+    } while (0)
 #define ROWS_FLUSH(base_index)                                                    \
     do {                                                                          \
         if (blockIdx.x == 0)                                                      \
@@ -53,6 +61,7 @@ __device__ long long g_rows_trace[32];
 #else
 #define ROWS_T0
 #define ROWS_T(i)
+#define ROWS_STAMP(i)
 #define ROWS_FLUSH(base_index)
 #endif
 
@@ -200,6 +209,7 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     // for this grid's completion before it reads a record
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
+    ROWS_STAMP(0);  // kernel start
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int split = static_cast<int>(blockIdx.x % p.num_splits);
     const int bh = static_cast<int>(blockIdx.x / p.num_splits);
@@ -253,6 +263,7 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem + C::kOffTmemSlot);
+    ROWS_STAMP(1);  // barriers, TMEM, CTA-wide sync done
 
     if (warp == kTmaWarp) {
         if (lane == 0) {
@@ -436,6 +447,8 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             }
             ROWS_T(7);
             wait_or_flag(bar(kBarSFull + s), (j >> 1) & 1, p.status);
+            if (j == 0) ROWS_STAMP(2);  // first scores ready
+            if (j == 1) ROWS_STAMP(3);  // second tile's scores ready
             ROWS_T(0);
             tc_fence_after();
             uint32_t a[RPT], g[RPT];
@@ -610,7 +623,9 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         if (threadIdx.x == 0) ROWS_FLUSH(0);
 
         // ---- row sums over the keys, then the epilogue: this thread's TMEM lane is head dimension kr ----
+        ROWS_STAMP(4);  // last weights handed over
         wait_or_flag(bar(kBarFinal), 0, p.status);
+        ROWS_STAMP(5);  // last value product done
         tc_fence_after();
         float* const dsum = reinterpret_cast<float*>(smem + C::kOffP);  // the weight tile is idle now: [8 warps][RPT][2], then [NR][2]
         {
@@ -672,12 +687,14 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         }
     }
 
+    ROWS_STAMP(6);  // epilogue stores issued
     tc_fence_before();
     __syncthreads();
     if (warp == kMmaWarp) {
         tc_fence_after();
         tmem_dealloc(tmem, C::kTmemCols);
     }
+    ROWS_STAMP(7);  // end
 }
 
 template <int NR, int HD>
