@@ -204,3 +204,43 @@ def test_rows_step_replayed_from_a_cuda_graph(plx, oracle):
     bits = {n: wl.bf16_bits(x[n]) for n in ("q", "r", "k", "v")}
     want, _ = oracle.prefill_bf16(bits["q"], bits["r"], bits["k"], bits["v"], None, cfg.scale)
     assert_parity(out.cpu().numpy(), want, torch.float32, "graph replay")
+
+
+@pytest.mark.parametrize("kind", ["peaked", "ascending", "probe_offset", "scale0", "negative_scale"])
+def test_rows_robustness_distributions(plx, oracle, kind):
+    """Inputs that stress the lazily moving references and the cancellation in the covariance branch, at sixteen rows
+    per KV head, one and eight splits: sharp distributions, scores that grow with every tile, a large common probe
+    component, a zero and a negative softmax scale."""
+    from parity_util import errors
+    Lq = 8
+    cfg = wl.DecodeConfig("rows rob", B=2, Hq=4, Hkv=2, D=128, T_max=2048, seed=3100)
+    x = wl.make_prefill_inputs(cfg, Lq, "cuda")
+    scale = cfg.scale
+    if kind == "peaked":
+        x["q"] = (x["q"].float() * 4).to(torch.bfloat16)
+    elif kind == "ascending":
+        for b in range(cfg.B):
+            for h in range(cfg.Hkv):
+                order = torch.argsort(x["k"][b, h].float() @ x["q"][b, h * cfg.G, 0].float())
+                x["k"][b, h] = x["k"][b, h][order]
+                x["v"][b, h] = x["v"][b, h][order]
+    elif kind == "probe_offset":
+        for b in range(cfg.B):
+            for h in range(cfg.Hkv):
+                rdir = x["r"][b, h * cfg.G, 0].float()
+                x["k"][b, h] = (x["k"][b, h].float() + 0.5 * rdir[None, :]).to(torch.bfloat16)
+    elif kind == "scale0":
+        scale = 0.0
+    elif kind == "negative_scale":
+        scale = -cfg.scale
+    bits = {n: wl.bf16_bits(x[n]) for n in ("q", "r", "k", "v")}
+    want, _ = oracle.prefill_bf16(bits["q"], bits["r"], bits["k"], bits["v"], None, scale)
+    ws = torch.empty(plx.parallax_prefill_workspace_bytes(cfg.B, cfg.Hq, cfg.D, Lq, 8), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for ns in (1, 8):
+        out = torch.full((cfg.B, cfg.Hq, Lq, cfg.D), float("nan"), dtype=torch.float32, device="cuda")
+        plx.parallax_decode_fwd_rows(x["q"], x["r"], x["k"], x["v"], None, out, scale, ws, ns, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        e = errors(out.cpu().numpy(), want)
+        assert e["rel_rms"] <= 1e-3 and e["max_abs"] <= 2e-2 * max(1.0, e["rms"]), (kind, ns, e)
