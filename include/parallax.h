@@ -378,7 +378,7 @@ int parallax_decode_fwd_multi(const void* q, const void* r, const void* k_cache,
  * PLX_ERR_DEVICE_TIMEOUT if a bounded device-side wait runs out.  PLX_ERR_UNSUPPORTED for other shapes.
  * parallax_decode_fwd_multi chooses this kernel by itself (parallax_decode_fwd_multi_paged too, over paged
  * caches); this entry forces it.  Arguments, token order and causal rule as parallax_decode_fwd_multi.  One or
- * two launches on `stream`; nothing is launched when an error is returned.
+ * two launches on `stream`; argument errors are returned before anything is launched.
  */
 int parallax_decode_fwd_rows(const void* q, const void* r, const void* k_cache, const void* v_cache,
                              const int32_t* seqlens, void* out, int B, int Hq, int Hkv, int D, int Lq,
