@@ -244,3 +244,15 @@ def test_rows_robustness_distributions(plx, oracle, kind):
         assert int(status.item()) == 0
         e = errors(out.cpu().numpy(), want)
         assert e["rel_rms"] <= 1e-3 and e["max_abs"] <= 2e-2 * max(1.0, e["rms"]), (kind, ns, e)
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("T", [1, 5, 17, 100])
+def test_rows_tiny_contexts(plx, oracle, D, T):
+    """Caches smaller than one 128-key tile (and than the tile's copy box), contexts shorter than the number of new
+    tokens: the tokens that see no key give rows of zeros."""
+    for Lq in (5, 16):
+        cfg = wl.DecodeConfig("rows tiny", B=1, Hq=2, Hkv=1, D=D, T_max=T, seed=3200 + T)
+        x, out = run_rows(plx, oracle, cfg, Lq, ns=1)
+        if T < Lq:   # token i sees T - (Lq - 1 - i) keys: the first Lq - T tokens see none
+            assert (out[:, :, :Lq - T] == 0).all()
