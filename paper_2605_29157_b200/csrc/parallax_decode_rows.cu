@@ -92,7 +92,9 @@ struct RowsCfg {
     static constexpr int kEwThreads = kEwWarps * 32;
     static constexpr int kMmaWarp = kEwWarps, kPvWarp = kEwWarps + 1, kTmaWarp = kEwWarps + 2;
     static constexpr int kThreads = (kEwWarps + 3) * 32;
-    static constexpr int kStagesK = HD == 64 ? 4 : NR == 16 ? 3 : 2, kStagesV = HD == 64 ? 4 : 3;
+    // ring depths by measurement (64 x 8192 keys, head dimension 64, 16 / 32 rows): K / V stages 4 / 4: 218 / 307 us, 3 / 3: 252 /
+    // 301, 2 / 3: 251 / 356, 6 / 6 (5 / 6 at 32 rows): 233 / 323 -- deeper rings than these are slower, not faster
+    static constexpr int kStagesK = HD == 64 ? (NR == 16 ? 4 : 3) : NR == 16 ? 3 : 2, kStagesV = HD == 64 ? (NR == 16 ? 4 : 3) : 3;
     static constexpr int kBoxQR = 2 * NR * 128;           // [Q rows; R rows] x 64 columns: the N = 2 NR operand of the score product
     static constexpr int kTileQR = kBoxes * kBoxQR;
     static constexpr int kPBlocks = 4 * NR / 64;          // 64-wide blocks of [P1 | P1 res | P2 | P2 res]
@@ -422,7 +424,10 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         float d1[RPT], d2[RPT];
 #pragma unroll
         for (int c = 0; c < RPT; ++c) d1[c] = d2[c] = 0.0f;
-        // bit c: row c0 + c exists (fewer than NR rows: the padding rows take part with weights of zero)
+        // bit c: row c0 + c exists.  With fewer than NR rows the padding rows (whatever the [Q; R] boxes hold past the
+        // last row: rows of the next head, or the zeros of the tensor map's bounds) are carried like real rows through
+        // the fully visible tiles (their columns of the weights and accumulators touch no other row's) and get weights
+        // of zero in the masked ones; nothing of them is stored
         const uint32_t row_mask = p.rows - c0 >= RPT ? (1u << RPT) - 1u : (p.rows > c0 ? (1u << (p.rows - c0)) - 1u : 0u);
         const float4* const ref4 = reinterpret_cast<const float4*>(ref + c0);
         ROWS_T0;
@@ -434,7 +439,7 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             const bool need_mask = (jt0 + j) * BK + BK > L - (p.Lq - 1);
             const uint32_t Sb = lane_base + C::kColS + s * 2 * NR;
             // bit c of vis: row c0 + c sees this thread's key (token i of a head sees the first L - (Lq - 1 - i) keys)
-            uint32_t vis = row_mask;
+            uint32_t vis = (1u << RPT) - 1u;
             if (need_mask) {
                 vis = 0u;
                 int tok = c0 % p.Lq;
@@ -459,9 +464,9 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             mbar_arrive(bar(kBarSFree + s));  // the score buffer is in registers
 
             // exponents against the references as they stand; does any visible score need a reference to move?
-            // `plain`: every row of this thread exists and sees every key of the tile (warp-uniform): packed
-            // arithmetic, no selects; a row without a reference yet gives x = +inf and raises the flag by itself
-            const bool plain = !need_mask && row_mask == (1u << RPT) - 1u;
+            // `plain`: every row sees every key of the tile (CTA-uniform): packed arithmetic, no selects; a row
+            // without a reference yet gives x = +inf and raises the flag by itself
+            const bool plain = !need_mask;
             float x[RPT];
             bool flag = false;
             if (plain) {

@@ -81,6 +81,34 @@ def test_rows_split_boundary_inside_the_new_tokens(plx, oracle):
         run_rows(plx, oracle, cfg, Lq, ns=(T + 127) // 128)
 
 
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("G,Lq", [(2, 5), (2, 12), (1, 9), (3, 7)])
+@pytest.mark.parametrize("ns", [1, 3])
+def test_rows_padding_rows_read_hostile_neighbours(plx, oracle, D, G, Lq, ns):
+    """Fewer rows than the tile holds: the padding rows of a CTA are whatever follows its rows in q and r (the next KV
+    head's, or nothing after the last one).  With NaN, infinities and huge values there, the rows of the head in front
+    must come out as if the neighbours were not there."""
+    T = 900
+    cfg = wl.DecodeConfig("rows hostile", B=2, Hq=3 * G, Hkv=3, D=D, T_max=T, seed=2450 + D + Lq)
+    x = wl.make_prefill_inputs(cfg, Lq, "cuda")
+    bits = {n: wl.bf16_bits(x[n]) for n in ("q", "r", "k", "v")}
+    want, _ = oracle.prefill_bf16(bits["q"], bits["r"], bits["k"], bits["v"], None, cfg.scale)
+    hostile = torch.tensor([float("nan"), float("inf"), -float("inf"), 3.0e38, -3.0e38, 1.0e4], device="cuda")
+    for name in ("q", "r"):   # the middle KV head's rows of both sequences
+        mid = x[name][:, G:2 * G]
+        mid.copy_(hostile[torch.arange(mid.numel(), device="cuda") % hostile.numel()].view(mid.shape).to(mid.dtype))
+    ws = torch.empty(plx.parallax_prefill_workspace_bytes(cfg.B, cfg.Hq, cfg.D, Lq, 8), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = torch.full((cfg.B, cfg.Hq, Lq, D), float("nan"), dtype=torch.float32, device="cuda")
+    plx.parallax_decode_fwd_rows(x["q"], x["r"], x["k"], x["v"], None, out, cfg.scale, ws, ns, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    got = out.cpu().numpy()
+    keep = [h for h in range(cfg.Hq) if not G <= h < 2 * G]
+    assert np.isfinite(got[:, keep]).all()
+    assert_parity(got[:, keep], want[:, keep], torch.float32, f"hostile neighbours D={D} G={G} Lq={Lq} ns={ns}")
+
+
 @pytest.mark.parametrize("Lq", [8, 14])
 @pytest.mark.parametrize("kind", ["peaked", "growing"])
 def test_rows_reference_moves_late(plx, oracle, kind, Lq):
