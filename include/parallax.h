@@ -139,7 +139,8 @@ int parallax_decode_plan(int B, int Hq, int Hkv, int D, int T_max, int num_sms, 
  *                    parallax_decode_workspace_bytes(B, Hq, D, splits used);
  *                    may be NULL only when the call resolves to one split.
  *                    Zero it once before first use (cudaMemset); every call leaves
- *                    the words it relies on (status, arrival counters) zero again.
+ *                    the words it relies on (status, the item ticket of the
+ *                    multi-token kernel, arrival counters) zero again.
  *                    Zero it again after a call that failed on the device.  Calls
  *                    that overlap on the GPU must not share a workspace.
  *   num_splits       0 = let the library plan; otherwise the number of key chunks
@@ -361,6 +362,9 @@ int parallax_decode_fwd_paged_fp8(const void* q, const void* r, const void* k_pa
  * workspace, so the call accepts any Lq.  (Steps of 9..64 rows whose q, r or out is not 16-byte
  * aligned stay on the decode kernel; parallax_decode_fwd_args always does.)  Workspace as parallax_decode_fwd_ex for Hq * Lq
  * query heads (parallax_decode_workspace_bytes(B, Hq * Lq, D, max_splits)); everything else as there.
+ * With a workspace, a step of nine to 32 rows per KV head and more (sequence, KV head, split) items
+ * than SMs runs one CTA per SM that draws its items from a word of the workspace's header (zero
+ * between calls, like the status word); without one it runs one CTA per item.
  */
 int parallax_decode_fwd_multi(const void* q, const void* r, const void* k_cache, const void* v_cache,
                               const int32_t* seqlens, void* out, int B, int Hq, int Hkv, int D, int Lq,

@@ -1737,6 +1737,13 @@ int parallax_decode_fwd_fp8(const void* q, const void* r, const void* k_cache, c
 #endif
 constexpr int kMultiTokenDecodeRows = PLX_MULTI_TOKEN_DECODE_ROWS;
 constexpr int kTwoCtaDecodeRows = 16;
+// The word of a decode workspace's header from which the CTAs of the multi-token tensor-core kernel draw their items
+// (zero between calls, like the status word in front of it).
+static int32_t* rows_ticket(void* workspace, size_t workspace_bytes)
+{
+    return (workspace && workspace_bytes >= kHeaderBytes) ? static_cast<int32_t*>(workspace) + 4 : nullptr;
+}
+
 // The part of a decode workspace that holds split records (after the status word, counters and staging).
 static void records_region(void* workspace, size_t workspace_bytes, int B, int rows, int D, void** rec, size_t* rec_bytes)
 {
@@ -1781,7 +1788,7 @@ int parallax_decode_fwd_multi(const void* q, const void* r, const void* k_cache,
         int32_t* status = (workspace && workspace_bytes >= kHeaderBytes) ? static_cast<int32_t*>(workspace) : nullptr;
         return plx_decode_rows_fwd(q, r, k_cache, v_cache, seqlens, out, B, Hq, Hkv, D, Lq, T_max, scale, out_dtype, rec,
                                    rec_bytes, rec ? num_splits : (num_splits > 1 ? 1 : num_splits), status,
-                                   static_cast<cudaStream_t>(stream), nullptr, 0, 0, 0);
+                                   static_cast<cudaStream_t>(stream), nullptr, 0, 0, 0, rows_ticket(workspace, workspace_bytes));
     }
     if (use_tensor_core_kernel(q, r, out, B, Hq, Hkv, Lq, D)) {
         void* rec = nullptr;
@@ -1884,7 +1891,8 @@ int parallax_decode_fwd_multi_paged(const void* q, const void* r, const void* k_
         int32_t* status = (workspace && workspace_bytes >= kHeaderBytes) ? static_cast<int32_t*>(workspace) : nullptr;
         return plx_decode_rows_fwd(q, r, k_pages, v_pages, seqlens, out, B, Hq, Hkv, D, Lq, static_cast<int>(T_cap), scale,
                                    out_dtype, rec, rec_bytes, rec ? num_splits : (num_splits > 1 ? 1 : num_splits), status,
-                                   static_cast<cudaStream_t>(stream), block_table, page_size, max_pages_per_seq, pool);
+                                   static_cast<cudaStream_t>(stream), block_table, page_size, max_pages_per_seq, pool,
+                                   rows_ticket(workspace, workspace_bytes));
     }
     if (page_size % 64 == 0 && use_tensor_core_kernel(q, r, out, B, Hq, Hkv, Lq, D)) {  // that kernel walks 64-key tiles
         void* rec = nullptr;

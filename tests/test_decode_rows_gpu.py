@@ -234,6 +234,75 @@ def test_rows_step_replayed_from_a_cuda_graph(plx, oracle):
     assert_parity(out.cpu().numpy(), want, torch.float32, "graph replay")
 
 
+def _sm_count():
+    return torch.cuda.get_device_properties(0).multi_processor_count
+
+
+@pytest.mark.parametrize("D,Lq,T,ns", [(128, 8, 600, 1), (128, 16, 900, 3), (64, 8, 700, 2), (64, 12, 400, 1)])
+def test_rows_more_items_than_sms_drawn_from_the_ticket(plx, oracle, D, Lq, T, ns):
+    """More (sequence, KV head, split) items than SMs through the routed entry with a zeroed workspace: one CTA per SM
+    draws items from the workspace's ticket word and carries its rings and barrier phases from item to item.  Equal
+    contexts and contexts of their own lengths (empty ones and ones shorter than the new tokens among them: items
+    without keys inside the walk); three calls in a row on the same workspace (the word is back at zero each time)
+    must agree bit for bit."""
+    Hkv = 8
+    B = (_sm_count() + Hkv * ns - 1) // (Hkv * ns) + 3          # a few items more than SMs, not a multiple of them
+    assert B * Hkv * ns > _sm_count()
+    cfg = wl.DecodeConfig("rows ticket", B=B, Hq=2 * Hkv, Hkv=Hkv, D=D, T_max=T, seed=3100 + D + Lq)
+    rng = np.random.default_rng(cfg.seed)
+    ragged = rng.integers(0, T + 1, size=B).astype(np.int32)
+    ragged[:4] = (0, Lq - 1, T, 1)
+    for seqlens in (None, ragged):
+        x = wl.make_prefill_inputs(cfg, Lq, "cuda")
+        if seqlens is not None:
+            x["seqlens"] = torch.from_numpy(seqlens).cuda()
+            for b in range(B):
+                x["k"][b, :, int(seqlens[b]):] = float("nan")
+                x["v"][b, :, int(seqlens[b]):] = float("nan")
+        bits = {n: wl.bf16_bits(x[n]) for n in ("q", "r", "k", "v")}
+        want, _ = oracle.prefill_bf16(bits["q"], bits["r"], bits["k"], bits["v"], seqlens, cfg.scale)
+        ws = plx.alloc_workspace(B, cfg.Hq * Lq, D, max(ns, 1), "cuda")
+        outs = []
+        for _ in range(3):
+            out = torch.full((B, cfg.Hq, Lq, D), float("nan"), dtype=torch.float32, device="cuda")
+            plx.parallax_decode_fwd_multi(x["q"], x["r"], x["k"], x["v"], x["seqlens"], out, cfg.scale, ws, ns)
+            torch.cuda.synchronize()
+            assert plx.parallax_workspace_status(ws) == 0
+            outs.append(out)
+        assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])
+        assert int(ws[:256].view(torch.int32).abs().sum().item()) == 0      # status and ticket are zero again
+        assert_parity(outs[0].cpu().numpy(), want, torch.float32, f"ticket D={D} Lq={Lq} ns={ns} ragged={seqlens is not None}")
+
+
+def test_rows_ticket_walk_over_a_paged_cache_and_from_a_cuda_graph(plx, oracle):
+    """The item walk over a paged cache (16-key pages), eager and replayed twice from a CUDA graph."""
+    Lq, T, page_size, Hkv = 8, 500, 16, 8
+    B = _sm_count() // Hkv + 5
+    cfg = wl.DecodeConfig("rows ticket paged", B=B, Hq=2 * Hkv, Hkv=Hkv, D=128, T_max=T, ragged=(Lq, T), seed=3200)
+    x = wl.make_prefill_inputs(cfg, Lq, "cuda")
+    kp, vp, table = wl.to_paged(x["k"], x["v"], page_size, seed=11)
+    bits = {n: wl.bf16_bits(x[n]) for n in ("q", "r", "k", "v")}
+    want, _ = oracle.prefill_bf16(bits["q"], bits["r"], bits["k"], bits["v"], x["seqlens_host"], cfg.scale)
+    ws = plx.alloc_workspace(B, cfg.Hq * Lq, cfg.D, 1, "cuda")
+    out = torch.full((B, cfg.Hq, Lq, cfg.D), float("nan"), dtype=torch.float32, device="cuda")
+    plx.parallax_decode_fwd_multi_paged(x["q"], x["r"], kp, vp, table, x["seqlens"], out, cfg.scale, ws, 1)
+    torch.cuda.synchronize()
+    assert plx.parallax_workspace_status(ws) == 0
+    assert_parity(out.cpu().numpy(), want, torch.float32, "ticket paged")
+    eager = out.clone()
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            plx.parallax_decode_fwd_multi_paged(x["q"], x["r"], kp, vp, table, x["seqlens"], out, cfg.scale, ws, 1, stream)
+    for _ in range(2):
+        out.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert plx.parallax_workspace_status(ws) == 0
+        assert torch.equal(out, eager)
+
+
 @pytest.mark.parametrize("kind", ["peaked", "ascending", "probe_offset", "scale0", "negative_scale"])
 def test_rows_robustness_distributions(plx, oracle, kind):
     """Inputs that stress the lazily moving references and the cancellation in the covariance branch, at sixteen rows
