@@ -1174,7 +1174,7 @@ plx_combine_kernel(const float* __restrict__ partials, const int32_t* __restrict
 // holding 2 D / 32 elements of O1 and O2.
 // ---------------------------------------------------------------------------
 constexpr int kRowCombineWarps = 8;
-constexpr int kRowCombineMaxSplits = 8;
+constexpr int kRowCombineMaxSplits = 16;
 
 template <int D>
 __global__ void __launch_bounds__(kRowCombineWarps * 32)
