@@ -836,6 +836,32 @@ bool plx_decode_rows_supported(int Hq, int Hkv, int D, int Lq)
 // Paged cache: block_table != nullptr, k_cache / v_cache are the page pools of pool_rows rows, T_max = page_size * max_pages.
 bool plx_decode_rows_page_size_ok(int page_size) { return page_size > 0 && page_size % 16 == 0 && (BK % page_size == 0 || page_size % BK == 0); }
 
+// Modelled time (us) of a step of `base` (sequence, KV head) pairs, each cut into c splits of a context of `tiles`
+// 128-key tiles, on `sms` SMs; used only to choose c.  The items run in generations of `sms`; a 128-key tile takes the
+// longer of the SM's own time for it (the element-wise chain: about 0.62 / 0.78 us at sixteen rows and D = 128 / 64,
+// 1.15 / 1.10 us at 32 rows) and its share of HBM (tile bytes x active SMs / 7 TB/s), so a last generation of few
+// items runs at the SM's pace while full ones run at HBM's; an item costs 1.2 us besides its tiles, a split step its
+// merge (5 us and the records written and read).  Fitted to and checked against measured steps of 20...128 sequences
+// of 2048...16384 keys (within 5 % on all of them but two, 8 % on those).
+static double rows_step_model(long long base, int sms, int tiles, int c, int nr, int D, long long rows, int page_box)
+{
+    const long long items = base * c;
+    const int tps = (tiles + c - 1) / c;
+    double t_sm = nr == 16 ? (D == 128 ? 0.62 : 0.78) : (D == 128 ? 1.15 : 1.10);
+    // small pages: the producer warp's copies per tile set the SM's pace (16-key pages: 1.6 us measured)
+    if (page_box > 0 && page_box <= 32 && t_sm < 25.6 / page_box) t_sm = 25.6 / page_box;
+    const double t_hbm = 2.0 * 128 * D * 2 * sms / 7.0e6;  // K and V tile, bf16, every SM streaming
+    const long long full = items / sms, rem = items % sms;
+    double t = static_cast<double>(full) * tps * (t_sm > t_hbm ? t_sm : t_hbm);
+    if (rem) {
+        const double share = t_hbm * static_cast<double>(rem) / sms;
+        t += tps * (t_sm > share ? t_sm : share);
+    }
+    t += 1.2 * static_cast<double>((items + sms - 1) / sms);
+    if (c > 1) t += 5.0 + 2.0 * static_cast<double>(rows) * c * (2 * D + 4) * 4 / 7.0e6;
+    return t;
+}
+
 int plx_decode_rows_fwd(const void* q, const void* r, const void* k_cache, const void* v_cache, const int32_t* seqlens,
                         void* out, int B, int Hq, int Hkv, int D, int Lq, int T_max, float scale, int out_dtype,
                         void* records, size_t record_bytes, int num_splits, int32_t* status, cudaStream_t stream,
@@ -870,8 +896,8 @@ int plx_decode_rows_fwd(const void* q, const void* r, const void* k_cache, const
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
         return PLX_ERR_CUDA;
     // Split plan (one CTA per SM is resident).  Fewer CTAs than SMs: as many splits as keep the grid within one
-    // generation, at least four 128-key tiles each.  More: the split count of 1..4 that wastes the least of the last
-    // generation, at least sixteen tiles each.  Always what the record space holds.
+    // generation, at least four 128-key tiles each.  More: the split count whose modelled time is least
+    // (rows_step_model), at least eight tiles each.  Always what the record space holds.
     const long long base_ctas = static_cast<long long>(B) * Hkv;
     const int tiles_max = (T_max + BK - 1) / BK;
     int ns = 1;
@@ -884,10 +910,10 @@ int plx_decode_rows_fwd(const void* q, const void* r, const void* k_cache, const
                 if (ns > 64) ns = 64;
             } else {
                 double best = 1e30;
-                for (int c = 1; c <= 4 && tiles_max / c >= 16; ++c) {
-                    const long long ctas = base_ctas * c;
-                    const double cost = static_cast<double>((ctas + sms - 1) / sms) / c * (1.0 + 0.02 * (c - 1));
-                    if (cost < best - 1e-9) {
+                for (const int c : {1, 2, 3, 4, 6, 8}) {
+                    if (c > 1 && tiles_max / c < 8) break;
+                    const double cost = rows_step_model(base_ctas, sms, tiles_max, c, nr, D, static_cast<long long>(q_rows), block_table ? page_box : 0);
+                    if (cost < best * 0.995) {  // a larger count has to pay for its records
                         best = cost;
                         ns = c;
                     }
