@@ -436,9 +436,9 @@ def run_ours(args, rank, world, local_rank):
         step(i)
     t_call = timer.run(step, args.steps)
     ms_per_step = t_call["ms_per_step"]
-    # one launch per call, except steps the library hands to the tensor-core kernel (more than eight rows per KV head)
+    # one launch per call, except steps the library hands to a tensor-core kernel and splits (kernel + merge)
     route = "decode" if args.fp8_kv else multi_token_route(cfg, Lq, args.page_size)
-    launches_per_step = (rows_kernel_launches(cfg, Lq, sms) if route == "rows" else
+    launches_per_step = (rows_kernel_launches(cfg, Lq, sms, args.page_size) if route == "rows" else
                          tensor_core_launches(cfg, Lq, sms) if route == "row-major" and not args.page_size else 1)
     value = whole_job_value(kv_bytes, world, ms_per_step)
     assert plx.parallax_workspace_status(ws) == 0, "device-side wait timed out"
@@ -545,7 +545,7 @@ def run_ours(args, rank, world, local_rank):
         by_bytes = roofline.get("read_probe", {}).get("GBps_by_call_bytes")
         result["other_configs"] = {n: quick_config(n, sampler, read_peak, by_bytes) for n in sorted(wl.CONFIGS) if n != args.workload}
         result["other_workloads"] = {n: quick_tensor_workload(n, local_rank) for n in ("P2", "T1")}
-        for new_tokens in (4, 8):   # multi-token decode steps on the headline shape: 8 and 16 rows per KV head
+        for new_tokens in (2, 4, 8):   # multi-token decode steps on the headline shape: 4, 8 and 16 rows per KV head
             result["other_workloads"][f"{args.workload}_new_tokens_{new_tokens}"] = quick_multi_token(args.workload, new_tokens,
                                                                                                    sampler, read_peak)
             torch.cuda.empty_cache()
@@ -559,41 +559,22 @@ def run_ours(args, rank, world, local_rank):
 
 
 def multi_token_route(cfg, Lq, page_size=0):
-    """Mirrors the library's routing of a multi-token step (only to name the kernel and count launches): up to
-    eight rows per KV head the decode kernel; nine to 32 rows the keys-on-lanes tensor-core kernel
-    ("rows"; paged caches when the page size divides 128 or is a multiple of it); otherwise nine to sixteen rows
-    that split into two CTAs of at most eight stay on the decode kernel and everything else goes to the row-major
-    tensor-core kernel."""
-    rows = cfg.G * Lq
-    if rows <= 8:
-        return "decode"
-    if rows <= 32 and cfg.D in (64, 128) and (not page_size or 128 % page_size == 0 or page_size % 128 == 0):
-        return "rows"
-    if rows <= 16:
-        g = max(c for c in range(1, 9) if rows % c == 0)
-        if rows // g <= 2:
-            return "decode"
-    return "row-major"
+    """The kernel the library runs for a multi-token step of this shape (asked of the library itself, only to name
+    the kernel and count launches): "decode", "rows" (keys-on-lanes tensor-core kernel) or "row-major"."""
+    from paper_2605_29157_b200 import binding as plx
+    kernel, _ = plx.parallax_decode_multi_plan(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, Lq, cfg.T_max, page_size)
+    return {plx.PLX_MULTI_KERNEL_DECODE: "decode", plx.PLX_MULTI_KERNEL_ROWS: "rows",
+            plx.PLX_MULTI_KERNEL_ROW_MAJOR: "row-major"}[kernel]
 
 
 def routed_to_tensor_core(cfg, Lq):
     return multi_token_route(cfg, Lq) != "decode"
 
 
-def rows_kernel_launches(cfg, Lq, sms):
-    """Launches per call of the keys-on-lanes kernel: 2 when the library splits the keys (kernel + merge), else 1.
-    Mirrors the library's plan only to count launches."""
-    base, tiles = cfg.B * cfg.Hkv, -(-cfg.T_max // 128)
-    if base < sms:
-        ns = min(sms // base, max(1, tiles // 4), 64)
-    else:
-        ns, best = 1, 1e30
-        for c in range(1, 5):
-            if tiles // c < 16:
-                break
-            cost = -(-base * c // sms) / c * (1.0 + 0.02 * (c - 1))
-            if cost < best - 1e-9:
-                best, ns = cost, c
+def rows_kernel_launches(cfg, Lq, sms, page_size=0):
+    """Launches per call of the keys-on-lanes kernel: 2 when the library splits the keys (kernel + merge), else 1."""
+    from paper_2605_29157_b200 import binding as plx
+    _, ns = plx.parallax_decode_multi_plan(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, Lq, cfg.T_max, page_size)
     return 2 if ns > 1 else 1
 
 

@@ -356,7 +356,7 @@ int parallax_decode_fwd_paged_fp8(const void* q, const void* r, const void* k_pa
  * query head are handled like Lq more query heads of its KV head (split-KV, fused merge and the
  * bandwidth-bound streaming of the decode kernel apply), so the call is HBM-bound where the
  * tensor-core multi-token kernel would compute a 128-row tile for a handful of rows.  That holds up
- * to eight rows per KV head (Lq * Hq / Hkv <= 8, one CTA per KV head).  Nine to 32 rows run
+ * to eight rows per KV head (Lq * Hq / Hkv <= 8, one CTA per KV head; four at D = 128).  Nine (five) to 32 rows run
  * on the tensor-core kernel of parallax_decode_fwd_rows (keys on the accumulator lanes), larger steps
  * on parallax_prefill_fwd_ex (residual weights); both keep their split records in the same
  * workspace, so the call accepts any Lq.  (Steps of 9..64 rows whose q, r or out is not 16-byte
@@ -388,6 +388,19 @@ int parallax_decode_fwd_rows(const void* q, const void* r, const void* k_cache, 
                              const int32_t* seqlens, void* out, int B, int Hq, int Hkv, int D, int Lq,
                              int T_max, float scale, int out_dtype, void* workspace, size_t workspace_bytes,
                              int num_splits, int32_t* status, void* stream);
+
+/*
+ * Which kernel parallax_decode_fwd_multi (page_size = 0) or parallax_decode_fwd_multi_paged would run for a step
+ * of this shape, given 16-byte aligned tensors and a workspace with room for split records, and, for the
+ * keys-on-lanes kernel, the split count it would plan for num_splits = 0 (1 = no merge launch; 0 is reported for
+ * the other kernels).  Host only: nothing is launched, no pointer is needed.  For callers that account for
+ * launches or want to log the route; the numbers follow the device the calling thread has current.
+ */
+#define PLX_MULTI_KERNEL_DECODE 0    /* the decode kernel: up to eight rows per KV head (four at D = 128) */
+#define PLX_MULTI_KERNEL_ROWS 1      /* the keys-on-lanes tensor-core kernel: up to 32 rows per KV head */
+#define PLX_MULTI_KERNEL_ROW_MAJOR 2 /* the row-major split-KV tensor-core kernel */
+int parallax_decode_multi_plan(int B, int Hq, int Hkv, int D, int Lq, int T_max, int page_size, int* kernel,
+                               int* num_splits);
 
 /* parallax_decode_fwd_multi over the paged cache of parallax_decode_fwd_paged (q, r, out [B, Hq, Lq, D]);
  * the hand-over to the keys-on-lanes kernel needs a page_size that divides 128 or is a multiple of it,

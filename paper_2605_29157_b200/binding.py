@@ -53,7 +53,7 @@ EXPORTS = (
     "parallax_decode_step", "parallax_decode_fwd_fp8_per_head", "parallax_decode_fwd_paged_fp8_per_head",
     "parallax_decode_fwd_multi", "parallax_prefill_workspace_bytes", "parallax_prefill_fwd_ex",
     "parallax_prefill_fwd_paged_ex", "parallax_decode_fwd_multi_paged", "parallax_decode_fwd_args",
-    "parallax_read_probe", "parallax_decode_fwd_rows",
+    "parallax_read_probe", "parallax_decode_fwd_rows", "parallax_decode_multi_plan",
 )
 TEST_HOOK_EXPORTS = ("plx_test_bounded_wait",)
 
@@ -107,6 +107,7 @@ def _load() -> ctypes.CDLL:
                                             vp, sz, i32, vp]),
         "parallax_read_probe": (i32, [vp, sz, vp, i32, i32, vp, vp]),
         "parallax_decode_fwd_rows": (i32, [vp] * 6 + [i32] * 6 + [f32, i32, vp, sz, i32, vp, vp]),
+        "parallax_decode_multi_plan": (i32, [i32] * 7 + [vp, vp]),
         "plx_test_bounded_wait": (i32, [vp, ctypes.c_uint32, vp, vp]),
     }
     for name, (res, args) in sig.items():
@@ -306,6 +307,18 @@ def parallax_prefill_fwd_ex(q, r, k_cache, v_cache, seqlens, out, scale, workspa
                                         int(p_precision), _ptr(workspace), ws_bytes, int(num_splits), _ptr(status),
                                         _stream(stream)))
     return out
+
+
+PLX_MULTI_KERNEL_DECODE, PLX_MULTI_KERNEL_ROWS, PLX_MULTI_KERNEL_ROW_MAJOR = 0, 1, 2
+
+
+def parallax_decode_multi_plan(B, Hq, Hkv, D, Lq, T_max, page_size=0):
+    """(kernel, num_splits) the multi-token entries would use for this shape: kernel is one of PLX_MULTI_KERNEL_*,
+    num_splits the planned split count of the keys-on-lanes kernel (0 for the other kernels)."""
+    kernel, ns = ctypes.c_int(0), ctypes.c_int(0)
+    _check(_lib.parallax_decode_multi_plan(int(B), int(Hq), int(Hkv), int(D), int(Lq), int(T_max), int(page_size),
+                                           ctypes.byref(kernel), ctypes.byref(ns)))
+    return kernel.value, ns.value
 
 
 def parallax_decode_fwd_rows(q, r, k_cache, v_cache, seqlens, out, scale, workspace=None, num_splits=0, status=None,

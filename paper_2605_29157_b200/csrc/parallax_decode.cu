@@ -1806,6 +1806,8 @@ int parallax_decode_fwd_fp8(const void* q, const void* r, const void* k_cache, c
 #endif
 constexpr int kMultiTokenDecodeRows = PLX_MULTI_TOKEN_DECODE_ROWS;
 constexpr int kTwoCtaDecodeRows = 16;
+// rows per KV head above which a multi-token step goes to the keys-on-lanes tensor-core kernel
+static int rows_kernel_from(int D) { return D == 128 ? 4 : kMultiTokenDecodeRows; }
 // The word of a decode workspace's header from which the CTAs of the multi-token tensor-core kernel draw their items
 // (zero between calls, like the status word in front of it).
 static int32_t* rows_ticket(void* workspace, size_t workspace_bytes)
@@ -1849,7 +1851,12 @@ int parallax_decode_fwd_multi(const void* q, const void* r, const void* k_cache,
     // 339 / 339; 1 x 32768 37 / 37 / 39 / 39 against 52 / 59 / 57 / 58.  (Up to eight rows the decode kernel stays ahead
     // or level at large batches: 64 x 8192, 2 / 4 / 8 rows: 298 / 300 / 314 against 324 / 329 / 340.)  At D = 64, same
     // shapes, 16 / 32 rows: 64 x 8192 222 / 308 against 309 / 570; 2 x 131072 98 / 132 against 152 / 267.
-    if (static_cast<long long>(Hq / Hkv) * Lq > kMultiTokenDecodeRows && plx_decode_rows_supported(Hq, Hkv, D, Lq) &&
+    // Since that kernel walks its items, merges with a warp per row and plans its splits by a step model, it is also
+    // ahead from five rows on at D = 128 (6 / 8 rows, decode kernel against it: 128 x 2048 167 / 168 against 159 / 159;
+    // 32 x 8192 164 / 166 against 154 / 155; 16 x 8192 90 / 92 against 82 / 82; 64 x 8192 and 2 x 131072 level; at four
+    // rows the decode kernel leads by 1-10 %); at D = 64 the decode kernel keeps everything up to eight rows (8 rows:
+    // 128 x 512 35 against 46, 8 x 8192 30 against 33, 64 x 8192 183 against 178).
+    if (static_cast<long long>(Hq / Hkv) * Lq > rows_kernel_from(D) && plx_decode_rows_supported(Hq, Hkv, D, Lq) &&
         aligned(q, 16) && aligned(r, 16) && aligned(out, 16) && aligned(k_cache, 16) && aligned(v_cache, 16)) {
         void* rec = nullptr;
         size_t rec_bytes = 0;
@@ -1937,6 +1944,27 @@ int parallax_decode_fwd_paged(const void* q, const void* r, const void* k_pages,
                            max_pages_per_seq, static_cast<uint64_t>(pool_rows));
 }
 
+int parallax_decode_multi_plan(int B, int Hq, int Hkv, int D, int Lq, int T_max, int page_size, int* kernel,
+                               int* num_splits)
+{
+    if (!kernel || !num_splits) return PLX_ERR_NULL_POINTER;
+    if (Lq <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || B <= 0 || T_max <= 0 || page_size < 0) return PLX_ERR_BAD_SHAPE;
+    const long long rows = static_cast<long long>(Hq / Hkv) * Lq;
+    const void* const aligned_ptr = reinterpret_cast<const void*>(static_cast<uintptr_t>(256));
+    *kernel = PLX_MULTI_KERNEL_DECODE;
+    *num_splits = 0;
+    const int from = (page_size == 0 || page_size >= 64) ? rows_kernel_from(D) : kMultiTokenDecodeRows;
+    if (rows > from && plx_decode_rows_supported(Hq, Hkv, D, Lq) && (page_size == 0 || plx_decode_rows_page_size_ok(page_size))) {
+        int sms = 0;
+        if (int rc = device_sm_count(&sms); rc != PLX_OK) return rc;
+        *kernel = PLX_MULTI_KERNEL_ROWS;
+        *num_splits = plx_decode_rows_plan(B, Hq, Hkv, D, Lq, T_max, page_size, sms);
+    } else if ((page_size == 0 || page_size % 64 == 0) && use_tensor_core_kernel(aligned_ptr, aligned_ptr, aligned_ptr, B, Hq, Hkv, Lq, D)) {
+        *kernel = PLX_MULTI_KERNEL_ROW_MAJOR;
+    }
+    return PLX_OK;
+}
+
 int parallax_decode_fwd_multi_paged(const void* q, const void* r, const void* k_pages, const void* v_pages,
                                     const int32_t* block_table, const int32_t* seqlens, void* out, int B, int Hq,
                                     int Hkv, int D, int Lq, int num_pages, int page_size, int max_pages_per_seq,
@@ -1948,7 +1976,9 @@ int parallax_decode_fwd_multi_paged(const void* q, const void* r, const void* k_
     if (workspace && !aligned(workspace, 16)) return PLX_ERR_ALIGNMENT;
     if (num_pages <= 0 || page_size <= 0 || page_size % kTileKeys != 0 || max_pages_per_seq <= 0)
         return PLX_ERR_BAD_SHAPE;
-    if (static_cast<long long>(Hq / Hkv) * Lq > kMultiTokenDecodeRows && plx_decode_rows_supported(Hq, Hkv, D, Lq) &&
+    // (small pages cost that kernel's producer sixteen or eight copies per tile: the earlier start only from 64-key pages on)
+    if (static_cast<long long>(Hq / Hkv) * Lq > (page_size >= 64 ? rows_kernel_from(D) : kMultiTokenDecodeRows) &&
+        plx_decode_rows_supported(Hq, Hkv, D, Lq) &&
         plx_decode_rows_page_size_ok(page_size) && aligned(q, 16) && aligned(r, 16) && aligned(out, 16) &&
         aligned(k_pages, 16) && aligned(v_pages, 16)) {  // nine to 32 rows per KV head: as in parallax_decode_fwd_multi
         const long long T_cap = static_cast<long long>(page_size) * max_pages_per_seq;

@@ -862,6 +862,34 @@ static double rows_step_model(long long base, int sms, int tiles, int c, int nr,
     return t;
 }
 
+// The split count the library plans for a call with room for its records (num_splits = 0).
+int plx_decode_rows_plan(int B, int Hq, int Hkv, int D, int Lq, int T_max, int page_size, int sms)
+{
+    const long long base_ctas = static_cast<long long>(B) * Hkv;
+    const int tiles_max = (T_max + BK - 1) / BK;
+    const int nr = (Hq / Hkv) * Lq <= 16 ? 16 : 32;
+    const int page_box = page_size > 0 ? (page_size < BK ? page_size : BK) : 0;
+    int ns = 1;
+    if (base_ctas < sms) {
+        const long long want = sms / base_ctas;
+        const long long most = tiles_max / 4 > 1 ? tiles_max / 4 : 1;
+        ns = static_cast<int>(want < most ? want : most);
+        if (ns > 64) ns = 64;
+    } else {
+        double best = 1e30;
+        for (const int c : {1, 2, 3, 4, 6, 8}) {
+            if (c > 1 && tiles_max / c < 8) break;
+            const double cost = rows_step_model(base_ctas, sms, tiles_max, c, nr, D, static_cast<long long>(B) * Hq * Lq, page_box);
+            if (cost < best * 0.995) {  // a larger count has to pay for its records
+                best = cost;
+                ns = c;
+            }
+        }
+    }
+    const int tps = (tiles_max + ns - 1) / ns;
+    return (tiles_max + tps - 1) / tps;  // no split without a tile
+}
+
 int plx_decode_rows_fwd(const void* q, const void* r, const void* k_cache, const void* v_cache, const int32_t* seqlens,
                         void* out, int B, int Hq, int Hkv, int D, int Lq, int T_max, float scale, int out_dtype,
                         void* records, size_t record_bytes, int num_splits, int32_t* status, cudaStream_t stream,
@@ -903,22 +931,7 @@ int plx_decode_rows_fwd(const void* q, const void* r, const void* k_cache, const
     int ns = 1;
     if (records) {
         if (num_splits == 0) {
-            if (base_ctas < sms) {
-                const long long want = sms / base_ctas;
-                const long long most = tiles_max / 4 > 1 ? tiles_max / 4 : 1;
-                ns = static_cast<int>(want < most ? want : most);
-                if (ns > 64) ns = 64;
-            } else {
-                double best = 1e30;
-                for (const int c : {1, 2, 3, 4, 6, 8}) {
-                    if (c > 1 && tiles_max / c < 8) break;
-                    const double cost = rows_step_model(base_ctas, sms, tiles_max, c, nr, D, static_cast<long long>(q_rows), block_table ? page_box : 0);
-                    if (cost < best * 0.995) {  // a larger count has to pay for its records
-                        best = cost;
-                        ns = c;
-                    }
-                }
-            }
+            ns = plx_decode_rows_plan(B, Hq, Hkv, D, Lq, T_max, block_table ? page_size : 0, sms);
         } else {
             ns = num_splits < tiles_max ? num_splits : tiles_max;
         }

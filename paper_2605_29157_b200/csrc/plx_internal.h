@@ -19,6 +19,7 @@ int plx_combine_after_producer(const float* partials, void* out, int rows, int D
 // calls of more items than SMs run one CTA per SM, each drawing (sequence, KV head, split) items from that word.
 bool plx_decode_rows_supported(int Hq, int Hkv, int D, int Lq);
 bool plx_decode_rows_page_size_ok(int page_size);
+int plx_decode_rows_plan(int B, int Hq, int Hkv, int D, int Lq, int T_max, int page_size, int sms);
 int plx_decode_rows_fwd(const void* q, const void* r, const void* k_cache, const void* v_cache, const int32_t* seqlens,
                         void* out, int B, int Hq, int Hkv, int D, int Lq, int T_max, float scale, int out_dtype,
                         void* records, size_t record_bytes, int num_splits, int32_t* status, cudaStream_t stream,

@@ -51,8 +51,9 @@ def test_default_line_has_every_section(cuda_device):
     d = _line("--workload", "C2", "--steps", "5", "--warmup", "3", "--cpu-seconds", "1")
     assert set(d["other_configs"]) == {"C1", "C3", "C4", "C5", "C6"}
     ow = d["other_workloads"]
-    assert {"P2", "T1", "C2_new_tokens_4", "C2_new_tokens_8"} <= set(ow)
-    assert ow["C2_new_tokens_8"]["kernel"] == "plx_decode_rows_kernel" and ow["C2_new_tokens_4"]["kernel"] == "plx_decode_kernel"
+    assert {"P2", "T1", "C2_new_tokens_2", "C2_new_tokens_4", "C2_new_tokens_8"} <= set(ow)
+    assert ow["C2_new_tokens_8"]["kernel"] == "plx_decode_rows_kernel" and ow["C2_new_tokens_2"]["kernel"] == "plx_decode_kernel"
+    assert ow["C2_new_tokens_4"]["kernel"] == "plx_decode_rows_kernel"      # eight rows per KV head at D = 128
     assert d["cpu_baseline"]["kind"] == "oracle" and d["sustained"]["value"] > 0
 
 

@@ -47,11 +47,14 @@ def test_args_entry_equals_the_specific_entries(plx):
                                  workspace=ws, num_splits=2)
     torch.cuda.synchronize()
     assert torch.equal(a, b)
-    # several tokens (eight rows per KV head: both entries use the decode kernel)
-    y = wl.make_prefill_inputs(cfg, 2, "cuda")
-    a4, b4 = new(cfg.B, cfg.Hq, 2, cfg.D), new(cfg.B, cfg.Hq, 2, cfg.D)
-    plx.parallax_decode_fwd_multi(y["q"], y["r"], y["k"], y["v"], y["seqlens"], a4, cfg.scale, ws, 0)
-    plx.parallax_decode_fwd_args(y["q"], y["r"], y["k"], y["v"], y["seqlens"], b4, cfg.scale, workspace=ws)
+    # several tokens (four rows per KV head: both entries use the decode kernel; from five rows on at this head dimension
+    # the routed entry hands the step to the keys-on-lanes kernel, which rounds differently)
+    cfg2 = wl.DecodeConfig("args multi", B=3, Hq=4, Hkv=2, D=128, T_max=1500, ragged=(2, 1500), seed=2301)
+    y = wl.make_prefill_inputs(cfg2, 2, "cuda")
+    assert plx.parallax_decode_multi_plan(cfg2.B, cfg2.Hq, cfg2.Hkv, cfg2.D, 2, cfg2.T_max)[0] == plx.PLX_MULTI_KERNEL_DECODE
+    a4, b4 = new(cfg2.B, cfg2.Hq, 2, cfg2.D), new(cfg2.B, cfg2.Hq, 2, cfg2.D)
+    plx.parallax_decode_fwd_multi(y["q"], y["r"], y["k"], y["v"], y["seqlens"], a4, cfg2.scale, ws, 0)
+    plx.parallax_decode_fwd_args(y["q"], y["r"], y["k"], y["v"], y["seqlens"], b4, cfg2.scale, workspace=ws)
     torch.cuda.synchronize()
     assert torch.equal(a4, b4)
 

@@ -164,3 +164,23 @@ def test_ten_to_sixteen_rows(plx, oracle, D, G, Lq):
     lens = g.integers(Lq, 701, size=B)
     lens[0], lens[1] = 700, Lq
     run_case(plx, oracle, cfg, Lq, ns=0, seqlens=lens)
+
+
+def test_the_plan_query_names_the_kernel_that_runs(plx):
+    """parallax_decode_multi_plan: the decode kernel up to four rows per KV head at D = 128 and up to eight at D = 64,
+    the keys-on-lanes kernel up to 32 rows (over pages only for page sizes it can tile; from five rows only over pages
+    of at least 64 keys), the row-major kernel above; a split count only for the keys-on-lanes kernel."""
+    K = plx
+    plan = lambda **kw: plx.parallax_decode_multi_plan(kw.get("B", 4), kw.get("Hq", 4), 2, kw.get("D", 128), kw["Lq"],
+                                                       kw.get("T", 4096), kw.get("ps", 0))
+    assert plan(Lq=1) == (K.PLX_MULTI_KERNEL_DECODE, 0) and plan(Lq=2)[0] == K.PLX_MULTI_KERNEL_DECODE
+    assert plan(Lq=3)[0] == K.PLX_MULTI_KERNEL_ROWS and plan(Lq=16)[0] == K.PLX_MULTI_KERNEL_ROWS
+    assert plan(Lq=17)[0] == K.PLX_MULTI_KERNEL_ROW_MAJOR and plan(Lq=200) == (K.PLX_MULTI_KERNEL_ROW_MAJOR, 0)
+    assert plan(Lq=4, D=64)[0] == K.PLX_MULTI_KERNEL_DECODE and plan(Lq=5, D=64)[0] == K.PLX_MULTI_KERNEL_ROWS
+    assert plan(Lq=3, ps=16)[0] == K.PLX_MULTI_KERNEL_DECODE and plan(Lq=3, ps=64)[0] == K.PLX_MULTI_KERNEL_ROWS
+    assert plan(Lq=8, ps=16)[0] == K.PLX_MULTI_KERNEL_ROWS and plan(Lq=8, ps=48)[0] != K.PLX_MULTI_KERNEL_ROWS
+    kernel, ns = plan(Lq=8, B=1, T=32768)         # two items on a whole GPU: split as far as four tiles per split allow
+    assert kernel == K.PLX_MULTI_KERNEL_ROWS and 2 <= ns <= 64
+    assert plan(Lq=8, B=256, T=2048) == (K.PLX_MULTI_KERNEL_ROWS, 1)
+    with pytest.raises(plx.ParallaxError):
+        plx.parallax_decode_multi_plan(4, 5, 2, 128, 1, 4096, 0)
