@@ -356,13 +356,14 @@ int parallax_decode_fwd_paged_fp8(const void* q, const void* r, const void* k_pa
  * query head are handled like Lq more query heads of its KV head (split-KV, fused merge and the
  * bandwidth-bound streaming of the decode kernel apply), so the call is HBM-bound where the
  * tensor-core multi-token kernel would compute a 128-row tile for a handful of rows.  That holds up
- * to eight rows per KV head (Lq * Hq / Hkv <= 8, one CTA per KV head; four at D = 128).  Nine (five) to 32 rows run
- * on the tensor-core kernel of parallax_decode_fwd_rows (keys on the accumulator lanes), larger steps
+ * to eight rows per KV head (Lq * Hq / Hkv <= 8, one CTA per KV head; four at D = 128).  Nine (five) to 64 rows run
+ * on the tensor-core kernel of parallax_decode_fwd_rows (keys on the accumulator lanes; 33 to 64 rows at D = 64
+ * only for contexts of at least 4096 keys on many sequences), larger steps
  * on parallax_prefill_fwd_ex (residual weights); both keep their split records in the same
  * workspace, so the call accepts any Lq.  (Steps of 9..64 rows whose q, r or out is not 16-byte
  * aligned stay on the decode kernel; parallax_decode_fwd_args always does.)  Workspace as parallax_decode_fwd_ex for Hq * Lq
  * query heads (parallax_decode_workspace_bytes(B, Hq * Lq, D, max_splits)); everything else as there.
- * With a workspace, a step of nine to 32 rows per KV head and more (sequence, KV head, split) items
+ * With a workspace, a step on that kernel with more (sequence, KV head, split) items
  * than SMs runs one CTA per SM that draws its items from a word of the workspace's header (zero
  * between calls, like the status word); without one it runs one CTA per item.
  */
@@ -374,7 +375,8 @@ int parallax_decode_fwd_multi(const void* q, const void* r, const void* k_cache,
 /*
  * The same step on the tensor-core kernel that keeps the KEYS on the accumulator lanes (Algorithm 1 with
  * S^T = K_c [Q; R]^T per 128-key tile and O^T += V_c^T P^T, so the tensor work follows the rows present):
- * up to 32 rows per KV head (Lq * Hq / Hkv <= 32), D = 64 or 128, bf16 caches, contiguous layout; q, r, k_cache,
+ * up to 64 rows per KV head (Lq * Hq / Hkv <= 64; more than 32 are worked as two halves that share their K/V
+ * through L2), D = 64 or 128, bf16 caches, contiguous layout; q, r, k_cache,
  * v_cache, out 16-byte aligned.  Split-KV like parallax_prefill_fwd_ex: `workspace` holds split records only
  * (parallax_prefill_workspace_bytes(B, Hq, D, Lq, max_splits) bytes, 16-byte aligned; NULL = one split),
  * num_splits 0 = planned (about one CTA per SM, at least four 128-key tiles per split), records merged by the
@@ -397,7 +399,7 @@ int parallax_decode_fwd_rows(const void* q, const void* r, const void* k_cache, 
  * launches or want to log the route; the numbers follow the device the calling thread has current.
  */
 #define PLX_MULTI_KERNEL_DECODE 0    /* the decode kernel: up to eight rows per KV head (four at D = 128) */
-#define PLX_MULTI_KERNEL_ROWS 1      /* the keys-on-lanes tensor-core kernel: up to 32 rows per KV head */
+#define PLX_MULTI_KERNEL_ROWS 1      /* the keys-on-lanes tensor-core kernel: up to 64 rows per KV head */
 #define PLX_MULTI_KERNEL_ROW_MAJOR 2 /* the row-major split-KV tensor-core kernel */
 int parallax_decode_multi_plan(int B, int Hq, int Hkv, int D, int Lq, int T_max, int page_size, int* kernel,
                                int* num_splits);

@@ -22,6 +22,8 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
+
+#include <algorithm>
 #include <math.h>
 #include <stdint.h>
 
@@ -1808,6 +1810,22 @@ constexpr int kMultiTokenDecodeRows = PLX_MULTI_TOKEN_DECODE_ROWS;
 constexpr int kTwoCtaDecodeRows = 16;
 // rows per KV head above which a multi-token step goes to the keys-on-lanes tensor-core kernel
 static int rows_kernel_from(int D) { return D == 128 ? 4 : kMultiTokenDecodeRows; }
+// Does a step of this shape go to the keys-on-lanes kernel (given that it supports the shape)?  page_size 0: contiguous.
+// 33 to 64 rows per KV head run there as two parts that share their K/V through L2: at D = 128 that beats the row-major
+// kernel everywhere measured (64 x 8192 keys 676-694 -> 539 us, 128 x 2048 333 -> 292, 16 x 8192 169 -> 146-156,
+// 2 x 131072 316-323 -> 280, 1 x 32768 56 -> 46); at D = 64 only long contexts on many sequences (64 x 8192 500 -> 422 us;
+// 128 x 2048, 16 x 8192 and 2 x 131072 lose 3-5 %).
+static bool rows_kernel_takes(int B, int Hq, int Hkv, int D, int Lq, int T_max, int page_size)
+{
+    const long long rows = static_cast<long long>(Hq / Hkv) * Lq;
+    const int from = (page_size == 0 || page_size >= 64) ? rows_kernel_from(D) : kMultiTokenDecodeRows;
+    if (rows <= from || !plx_decode_rows_supported(Hq, Hkv, D, Lq)) return false;
+    if (page_size != 0 && !plx_decode_rows_page_size_ok(page_size)) return false;
+    if (rows <= 32 || D == 128) return true;
+    int sms = 0;
+    if (device_sm_count(&sms) != PLX_OK) return false;
+    return T_max >= 32 * 128 && 2LL * B * Hkv >= 3LL * sms;
+}
 // The word of a decode workspace's header from which the CTAs of the multi-token tensor-core kernel draw their items
 // (zero between calls, like the status word in front of it).
 static int32_t* rows_ticket(void* workspace, size_t workspace_bytes)
@@ -1856,7 +1874,7 @@ int parallax_decode_fwd_multi(const void* q, const void* r, const void* k_cache,
     // 32 x 8192 164 / 166 against 154 / 155; 16 x 8192 90 / 92 against 82 / 82; 64 x 8192 and 2 x 131072 level; at four
     // rows the decode kernel leads by 1-10 %); at D = 64 the decode kernel keeps everything up to eight rows (8 rows:
     // 128 x 512 35 against 46, 8 x 8192 30 against 33, 64 x 8192 183 against 178).
-    if (static_cast<long long>(Hq / Hkv) * Lq > rows_kernel_from(D) && plx_decode_rows_supported(Hq, Hkv, D, Lq) &&
+    if (rows_kernel_takes(B, Hq, Hkv, D, Lq, T_max, 0) &&
         aligned(q, 16) && aligned(r, 16) && aligned(out, 16) && aligned(k_cache, 16) && aligned(v_cache, 16)) {
         void* rec = nullptr;
         size_t rec_bytes = 0;
@@ -1949,12 +1967,10 @@ int parallax_decode_multi_plan(int B, int Hq, int Hkv, int D, int Lq, int T_max,
 {
     if (!kernel || !num_splits) return PLX_ERR_NULL_POINTER;
     if (Lq <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || B <= 0 || T_max <= 0 || page_size < 0) return PLX_ERR_BAD_SHAPE;
-    const long long rows = static_cast<long long>(Hq / Hkv) * Lq;
     const void* const aligned_ptr = reinterpret_cast<const void*>(static_cast<uintptr_t>(256));
     *kernel = PLX_MULTI_KERNEL_DECODE;
     *num_splits = 0;
-    const int from = (page_size == 0 || page_size >= 64) ? rows_kernel_from(D) : kMultiTokenDecodeRows;
-    if (rows > from && plx_decode_rows_supported(Hq, Hkv, D, Lq) && (page_size == 0 || plx_decode_rows_page_size_ok(page_size))) {
+    if (rows_kernel_takes(B, Hq, Hkv, D, Lq, T_max, page_size)) {
         int sms = 0;
         if (int rc = device_sm_count(&sms); rc != PLX_OK) return rc;
         *kernel = PLX_MULTI_KERNEL_ROWS;
@@ -1977,10 +1993,11 @@ int parallax_decode_fwd_multi_paged(const void* q, const void* r, const void* k_
     if (num_pages <= 0 || page_size <= 0 || page_size % kTileKeys != 0 || max_pages_per_seq <= 0)
         return PLX_ERR_BAD_SHAPE;
     // (small pages cost that kernel's producer sixteen or eight copies per tile: the earlier start only from 64-key pages on)
-    if (static_cast<long long>(Hq / Hkv) * Lq > (page_size >= 64 ? rows_kernel_from(D) : kMultiTokenDecodeRows) &&
-        plx_decode_rows_supported(Hq, Hkv, D, Lq) &&
-        plx_decode_rows_page_size_ok(page_size) && aligned(q, 16) && aligned(r, 16) && aligned(out, 16) &&
-        aligned(k_pages, 16) && aligned(v_pages, 16)) {  // nine to 32 rows per KV head: as in parallax_decode_fwd_multi
+    if (rows_kernel_takes(B, Hq, Hkv, D, Lq,
+                          static_cast<int>(std::min<long long>(static_cast<long long>(page_size) * max_pages_per_seq, 0x7fffffff)),
+                          page_size) &&
+        aligned(q, 16) && aligned(r, 16) && aligned(out, 16) && aligned(k_pages, 16) &&
+        aligned(v_pages, 16)) {  // as in parallax_decode_fwd_multi
         const long long T_cap = static_cast<long long>(page_size) * max_pages_per_seq;
         const long long pool = static_cast<long long>(num_pages) * Hkv * page_size;
         if (T_cap >= (1LL << 31) - 65536 || pool >= (1LL << 31) - 65536) return PLX_ERR_BAD_SHAPE;

@@ -68,7 +68,7 @@ __device__ long long g_rows_trace[32];
 namespace {
 
 constexpr int BK = 128;  // keys per tile = TMEM lanes
-constexpr int kMaxRows = 32;
+constexpr int kMaxRows = 64;  // per KV head; more than 32 are worked as two parts (two items that share their K/V through L2)
 constexpr int kRowsPerThread = 8;              // rows per element-wise thread: NR / 8 threads share a key
 constexpr int kBoxKV = BK * 128;       // [128 keys x 64 columns] bf16 box: 16 KiB (a K or V tile is HD / 64 of them)
 constexpr int kBlockP = BK * 128;      // [128 keys x 64 columns of the stacked weights] bf16: 16 KiB
@@ -124,9 +124,10 @@ struct RowsParams {
     float* partials;   // nullptr: one split, rows finished here
     int32_t* status;
     int B, Hq, Hkv, Lq, T_max;
-    int rows;          // (Hq / Hkv) * Lq <= NR rows of a KV head, contiguous in [B, Hq, Lq, D]
+    int rows;          // (Hq / Hkv) * Lq rows of a KV head, contiguous in [B, Hq, Lq, D]
+    int parts, rows_per_part;  // the rows of a KV head are worked in `parts` items of at most rows_per_part <= NR rows
     int num_splits, tiles_per_split;
-    int n_items;       // B * Hkv * num_splits (sequence, KV head, key split) items
+    int n_items;       // B * Hkv * num_splits * parts (sequence, KV head, key split, part) items; parts of a split are neighbours
     // Device int32, zero between calls: the next item to hand out (the CTAs of a grid smaller than n_items draw their
     // items from it; the last draw of a launch sets it back to zero).  nullptr: one CTA per item.
     int32_t* ticket;
@@ -209,12 +210,17 @@ __device__ __forceinline__ void store_value(void* out, size_t idx, float v, int 
 // final / free pair per item.
 struct RowsItem {
     int b, hkv, split, L, jt0, n_tiles;
+    int row_off, rows;  // this item's rows of the KV head: row_off ... row_off + rows - 1
     size_t row0, kv_row0;
 };
 
 __device__ __forceinline__ RowsItem rows_item(const RowsParams& p, int item)
 {
     RowsItem it;
+    const int part = item % p.parts;
+    item /= p.parts;
+    it.row_off = part * p.rows_per_part;
+    it.rows = min(p.rows_per_part, p.rows - it.row_off);
     it.split = item % p.num_splits;
     const int bh = item / p.num_splits;
     it.b = bh / p.Hkv;
@@ -222,7 +228,7 @@ __device__ __forceinline__ RowsItem rows_item(const RowsParams& p, int item)
     const int G = p.Hq / p.Hkv;
     int L = p.seqlens ? p.seqlens[it.b] : p.T_max;
     it.L = max(0, min(L, p.T_max));
-    it.row0 = (static_cast<size_t>(it.b) * p.Hq + static_cast<size_t>(it.hkv) * G) * p.Lq;  // first row of this KV head
+    it.row0 = (static_cast<size_t>(it.b) * p.Hq + static_cast<size_t>(it.hkv) * G) * p.Lq + it.row_off;  // first row of this item
     it.kv_row0 = (static_cast<size_t>(it.b) * p.Hkv + it.hkv) * p.T_max;
     const int n_all = (it.L + BK - 1) / BK;
     it.jt0 = it.split * p.tiles_per_split;
@@ -500,11 +506,6 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         const int c0 = RPT * part;  // first row of this thread's columns
         const uint32_t lane_base = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
         const int swz = kr & 7;
-        // bit c: row c0 + c exists.  With fewer than NR rows the padding rows (whatever the [Q; R] boxes hold past the
-        // last row: rows of the next head, or the zeros of the tensor map's bounds) are carried like real rows through
-        // the fully visible tiles (their columns of the weights and accumulators touch no other row's) and get weights
-        // of zero in the masked ones; nothing of them is stored
-        const uint32_t row_mask = p.rows - c0 >= RPT ? (1u << RPT) - 1u : (p.rows > c0 ? (1u << (p.rows - c0)) - 1u : 0u);
         const float4* const ref4 = reinterpret_cast<const float4*>(ref + c0);
         int n = 0, g = 0;
         ROWS_T0;
@@ -515,12 +516,17 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             const RowsItem it = rows_item(p, item);
             const int L = it.L, jt0 = it.jt0, n_tiles = it.n_tiles;
             const size_t row0 = it.row0;
+            // bit c: row c0 + c exists.  With fewer than NR rows the padding rows (whatever the [Q; R] boxes hold past the
+            // last row: the next part's or the next head's rows, or the zeros of the tensor map's bounds) are carried like
+            // real rows through the fully visible tiles (their columns of the weights and accumulators touch no other
+            // row's) and get weights of zero in the masked ones; nothing of them is stored
+            const uint32_t row_mask = it.rows - c0 >= RPT ? (1u << RPT) - 1u : (it.rows > c0 ? (1u << (it.rows - c0)) - 1u : 0u);
             if (n_tiles == 0) {  // no key for this split: empty records (only m is ever read), or rows of zeros
                 if (p.partials) {
-                    for (int i = threadIdx.x; i < p.rows; i += kEwThreads)
+                    for (int i = threadIdx.x; i < it.rows; i += kEwThreads)
                         p.partials[((row0 + i) * p.num_splits + it.split) * REC] = -INFINITY;
                 } else {
-                    for (int i = threadIdx.x; i < p.rows * HD; i += kEwThreads) store_value(p.out, row0 * HD + i, 0.0f, p.out_dtype);
+                    for (int i = threadIdx.x; i < it.rows * HD; i += kEwThreads) store_value(p.out, row0 * HD + i, 0.0f, p.out_dtype);
                 }
                 continue;
             }
@@ -542,7 +548,7 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 uint32_t vis = (1u << RPT) - 1u;
                 if (need_mask) {
                     vis = 0u;
-                    int tok = c0 % p.Lq;
+                    int tok = (it.row_off + c0) % p.Lq;
 #pragma unroll
                     for (int c = 0; c < RPT; ++c) {
                         if (key < L - (p.Lq - 1 - tok)) vis |= 1u << c;
@@ -843,14 +849,15 @@ bool plx_decode_rows_page_size_ok(int page_size) { return page_size > 0 && page_
 // items runs at the SM's pace while full ones run at HBM's; an item costs 1.2 us besides its tiles, a split step its
 // merge (5 us and the records written and read).  Fitted to and checked against measured steps of 20...128 sequences
 // of 2048...16384 keys (within 5 % on all of them but two, 8 % on those).
-static double rows_step_model(long long base, int sms, int tiles, int c, int nr, int D, long long rows, int page_box)
+static double rows_step_model(long long base, int sms, int tiles, int c, int nr, int D, long long rows, int page_box, int parts)
 {
     const long long items = base * c;
     const int tps = (tiles + c - 1) / c;
     double t_sm = nr == 16 ? (D == 128 ? 0.62 : 0.78) : (D == 128 ? 1.15 : 1.10);
     // small pages: the producer warp's copies per tile set the SM's pace (16-key pages: 1.6 us measured)
     if (page_box > 0 && page_box <= 32 && t_sm < 25.6 / page_box) t_sm = 25.6 / page_box;
-    const double t_hbm = 2.0 * 128 * D * 2 * sms / 7.0e6;  // K and V tile, bf16, every SM streaming
+    // K and V tile, bf16, every SM streaming; the parts of a KV head's rows run side by side and share their tiles in L2
+    const double t_hbm = 2.0 * 128 * D * 2 * sms / 7.0e6 / parts;
     const long long full = items / sms, rem = items % sms;
     double t = static_cast<double>(full) * tps * (t_sm > t_hbm ? t_sm : t_hbm);
     if (rem) {
@@ -865,9 +872,11 @@ static double rows_step_model(long long base, int sms, int tiles, int c, int nr,
 // The split count the library plans for a call with room for its records (num_splits = 0).
 int plx_decode_rows_plan(int B, int Hq, int Hkv, int D, int Lq, int T_max, int page_size, int sms)
 {
-    const long long base_ctas = static_cast<long long>(B) * Hkv;
+    const int rows = (Hq / Hkv) * Lq;
+    const int parts = rows > 32 ? 2 : 1, rows_per_part = (rows + parts - 1) / parts;
+    const long long base_ctas = static_cast<long long>(B) * Hkv * parts;
     const int tiles_max = (T_max + BK - 1) / BK;
-    const int nr = (Hq / Hkv) * Lq <= 16 ? 16 : 32;
+    const int nr = rows_per_part <= 16 ? 16 : 32;
     const int page_box = page_size > 0 ? (page_size < BK ? page_size : BK) : 0;
     int ns = 1;
     if (base_ctas < sms) {
@@ -879,7 +888,7 @@ int plx_decode_rows_plan(int B, int Hq, int Hkv, int D, int Lq, int T_max, int p
         double best = 1e30;
         for (const int c : {1, 2, 3, 4, 6, 8}) {
             if (c > 1 && tiles_max / c < 8) break;
-            const double cost = rows_step_model(base_ctas, sms, tiles_max, c, nr, D, static_cast<long long>(B) * Hq * Lq, page_box);
+            const double cost = rows_step_model(base_ctas, sms, tiles_max, c, nr, D, static_cast<long long>(B) * Hq * Lq, page_box, parts);
             if (cost < best * 0.995) {  // a larger count has to pay for its records
                 best = cost;
                 ns = c;
@@ -908,8 +917,11 @@ int plx_decode_rows_fwd(const void* q, const void* r, const void* k_cache, const
     if (!plx_aligned(q, 16) || !plx_aligned(r, 16) || !plx_aligned(k_cache, 16) || !plx_aligned(v_cache, 16) ||
         !plx_aligned(out, 16) || (records && !plx_aligned(records, 16)))
         return PLX_ERR_ALIGNMENT;
+    // more than 32 rows per KV head: two items of half the rows each, neighbours in the item order, so that they run at
+    // the same time on two SMs and the second one's K/V tiles come out of L2
     const int rows = (Hq / Hkv) * Lq;
-    const int nr = rows <= 16 ? 16 : 32;
+    const int parts = rows > 32 ? 2 : 1, rows_per_part = (rows + parts - 1) / parts;
+    const int nr = rows_per_part <= 16 ? 16 : 32;
 
     CUtensorMap tmQ, tmR, tmK, tmV;
     int rc;
@@ -926,7 +938,7 @@ int plx_decode_rows_fwd(const void* q, const void* r, const void* k_cache, const
     // Split plan (one CTA per SM is resident).  Fewer CTAs than SMs: as many splits as keep the grid within one
     // generation, at least four 128-key tiles each.  More: the split count whose modelled time is least
     // (rows_step_model), at least eight tiles each.  Always what the record space holds.
-    const long long base_ctas = static_cast<long long>(B) * Hkv;
+    const long long base_ctas = static_cast<long long>(B) * Hkv * parts;
     const int tiles_max = (T_max + BK - 1) / BK;
     int ns = 1;
     if (records) {
@@ -943,7 +955,7 @@ int plx_decode_rows_fwd(const void* q, const void* r, const void* k_cache, const
     ns = (tiles_max + tps - 1) / tps;  // no split without a tile
     if (base_ctas * ns > 0x7fffffffLL) return PLX_ERR_BAD_SHAPE;
     RowsParams rp{seqlens, out, ns > 1 ? static_cast<float*>(records) : nullptr, status, B, Hq, Hkv, Lq, T_max,
-                  rows, ns, tps, static_cast<int>(base_ctas * ns), ticket, scale * 1.4426950408889634f, out_dtype, block_table,
+                  rows, parts, rows_per_part, ns, tps, static_cast<int>(base_ctas * ns), ticket, scale * 1.4426950408889634f, out_dtype, block_table,
                   page_size, max_pages, page_box, pool_rows};
     PlxNvtxRange nvtx_range("plx_decode_rows_fwd");
     // With a ticket word and more items than SMs: one CTA per SM, each drawing items until none is left (item i of a CTA

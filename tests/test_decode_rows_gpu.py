@@ -146,6 +146,51 @@ def test_rows_head_dimension_64(plx, oracle, G, Lq, T):
         run_rows(plx, oracle, cfg, Lq, ns=3, seqlens=[max(1, Lq - 1), 777], label="ragged")
 
 
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("G,Lq", [(2, 17), (2, 24), (2, 32), (4, 12), (1, 33), (8, 8), (3, 11), (1, 64)])
+@pytest.mark.parametrize("T,ns", [(128, 1), (300, 1), (1000, 3)])
+def test_rows_thirty_three_to_sixty_four_rows_in_two_parts(plx, oracle, D, G, Lq, T, ns):
+    """More than 32 rows per KV head: two items of half the rows each (the second part's tokens start in the middle of
+    a head's tokens, or with another head), one split and three, full and ragged last tiles."""
+    cfg = wl.DecodeConfig("rows parts", B=2, Hq=2 * G, Hkv=2, D=D, T_max=T, seed=3300 + G * Lq + T)
+    run_rows(plx, oracle, cfg, Lq, ns=ns)
+
+
+def test_rows_two_parts_ragged_paged_and_walked(plx, oracle):
+    """48 rows per KV head over contexts of their own lengths (empty, shorter than the new tokens, one key), through the
+    routed entry: contiguous with more items than SMs (the ticket walk over parts) and over 64-key pages."""
+    Lq, T, Hkv = 24, 700, 8
+    B = torch.cuda.get_device_properties(0).multi_processor_count // (2 * Hkv) + 2
+    cfg = wl.DecodeConfig("rows parts walk", B=B, Hq=2 * Hkv, Hkv=Hkv, D=128, T_max=T, seed=3400)
+    x = wl.make_prefill_inputs(cfg, Lq, "cuda")
+    rng = np.random.default_rng(5)
+    sl = rng.integers(0, T + 1, size=B).astype(np.int32)
+    sl[:4] = (0, Lq - 1, 1, T)
+    x["seqlens"] = torch.from_numpy(sl).cuda()
+    for b in range(B):
+        x["k"][b, :, int(sl[b]):] = float("nan")
+        x["v"][b, :, int(sl[b]):] = float("nan")
+    bits = {n: wl.bf16_bits(x[n]) for n in ("q", "r", "k", "v")}
+    want, _ = oracle.prefill_bf16(bits["q"], bits["r"], bits["k"], bits["v"], sl, cfg.scale)
+    assert plx.parallax_decode_multi_plan(B, cfg.Hq, Hkv, 128, Lq, T)[0] == plx.PLX_MULTI_KERNEL_ROWS
+    ws = plx.alloc_workspace(B, cfg.Hq * Lq, cfg.D, 4, "cuda")
+    for ns in (1, 2):
+        out = torch.full((B, cfg.Hq, Lq, cfg.D), float("nan"), dtype=torch.float32, device="cuda")
+        plx.parallax_decode_fwd_multi(x["q"], x["r"], x["k"], x["v"], x["seqlens"], out, cfg.scale, ws, ns)
+        torch.cuda.synchronize()
+        assert plx.parallax_workspace_status(ws) == 0
+        assert int(ws[:256].view(torch.int32).abs().sum().item()) == 0
+        assert_parity(out.cpu().numpy(), want, torch.float32, f"two parts walked ns={ns}")
+    x["k"].nan_to_num_(0.0)
+    x["v"].nan_to_num_(0.0)
+    kp, vp, table = wl.to_paged(x["k"], x["v"], 64, seed=3)
+    out = torch.full((B, cfg.Hq, Lq, cfg.D), float("nan"), dtype=torch.float32, device="cuda")
+    plx.parallax_decode_fwd_multi_paged(x["q"], x["r"], kp, vp, table, x["seqlens"], out, cfg.scale, ws, 0)
+    torch.cuda.synchronize()
+    assert plx.parallax_workspace_status(ws) == 0
+    assert_parity(out.cpu().numpy(), want, torch.float32, "two parts paged")
+
+
 def test_rows_rejects_what_it_does_not_serve(plx):
     q = torch.zeros(1, 4, 40, 128, dtype=torch.bfloat16, device="cuda")      # 80 rows per KV head
     k = torch.zeros(1, 2, 256, 128, dtype=torch.bfloat16, device="cuda")

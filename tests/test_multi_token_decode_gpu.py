@@ -168,14 +168,17 @@ def test_ten_to_sixteen_rows(plx, oracle, D, G, Lq):
 
 def test_the_plan_query_names_the_kernel_that_runs(plx):
     """parallax_decode_multi_plan: the decode kernel up to four rows per KV head at D = 128 and up to eight at D = 64,
-    the keys-on-lanes kernel up to 32 rows (over pages only for page sizes it can tile; from five rows only over pages
-    of at least 64 keys), the row-major kernel above; a split count only for the keys-on-lanes kernel."""
+    the keys-on-lanes kernel up to 64 rows (over pages only for page sizes it can tile; from five rows only over pages
+    of at least 64 keys; 33 to 64 rows at D = 64 only for long contexts on many sequences), the row-major kernel above; a split count only for the keys-on-lanes kernel."""
     K = plx
     plan = lambda **kw: plx.parallax_decode_multi_plan(kw.get("B", 4), kw.get("Hq", 4), 2, kw.get("D", 128), kw["Lq"],
                                                        kw.get("T", 4096), kw.get("ps", 0))
     assert plan(Lq=1) == (K.PLX_MULTI_KERNEL_DECODE, 0) and plan(Lq=2)[0] == K.PLX_MULTI_KERNEL_DECODE
     assert plan(Lq=3)[0] == K.PLX_MULTI_KERNEL_ROWS and plan(Lq=16)[0] == K.PLX_MULTI_KERNEL_ROWS
-    assert plan(Lq=17)[0] == K.PLX_MULTI_KERNEL_ROW_MAJOR and plan(Lq=200) == (K.PLX_MULTI_KERNEL_ROW_MAJOR, 0)
+    assert plan(Lq=17)[0] == K.PLX_MULTI_KERNEL_ROWS and plan(Lq=32)[0] == K.PLX_MULTI_KERNEL_ROWS    # two parts of 17 / 32 rows
+    assert plan(Lq=33)[0] == K.PLX_MULTI_KERNEL_ROW_MAJOR and plan(Lq=200) == (K.PLX_MULTI_KERNEL_ROW_MAJOR, 0)
+    assert plan(Lq=20, D=64)[0] == K.PLX_MULTI_KERNEL_ROW_MAJOR           # at D = 64 only long contexts on many sequences
+    assert plan(Lq=20, D=64, B=128, T=8192)[0] == K.PLX_MULTI_KERNEL_ROWS
     assert plan(Lq=4, D=64)[0] == K.PLX_MULTI_KERNEL_DECODE and plan(Lq=5, D=64)[0] == K.PLX_MULTI_KERNEL_ROWS
     assert plan(Lq=3, ps=16)[0] == K.PLX_MULTI_KERNEL_DECODE and plan(Lq=3, ps=64)[0] == K.PLX_MULTI_KERNEL_ROWS
     assert plan(Lq=8, ps=16)[0] == K.PLX_MULTI_KERNEL_ROWS and plan(Lq=8, ps=48)[0] != K.PLX_MULTI_KERNEL_ROWS
