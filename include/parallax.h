@@ -35,8 +35,9 @@
  *     expected to be in the cache already and counted by seqlens.
  *   - Supported shapes: D in {64, 128}; Hq a multiple of Hkv with group size
  *     Hq/Hkv from 1 to 64 (up to eight query heads of a KV head are served by one CTA;
- *     larger groups by several CTAs per KV head, or -- parallax_decode_fwd_ex and
- *     parallax_decode_fwd_paged route them by measured crossover -- by the tensor-core kernel,
+ *     larger groups by several CTAs per KV head, or -- parallax_decode_fwd_ex,
+ *     parallax_decode_fwd_paged and parallax_decode_step route them by measured crossover,
+ *     at D = 128 from five heads per KV head on -- by the tensor-core kernels,
  *     see parallax_decode_fwd_multi, which also lifts the limit of 64); q, r, out 4-byte
  *     aligned; k_cache, v_cache 16-byte aligned; workspace 16-byte aligned.
  *   - Launch ordering: the decode kernels are launched with the programmatic stream

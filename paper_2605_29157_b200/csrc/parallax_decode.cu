@@ -1757,6 +1757,8 @@ static int decode_fwd_impl(const void* q, const void* r, const void* k_cache, co
     return dispatch_main(D, g, tmK, tmV, kp, st, fp8);
 }
 
+constexpr int kMaxGroupOneCta = 8;  // query heads per KV head one CTA of the decode kernel serves (= PLX_MULTI_TOKEN_DECODE_ROWS)
+
 int parallax_decode_step(const void* q_raw, const void* r_raw, const void* k_raw, const void* v_raw,
                          const void* q_weight, const void* r_weight, const void* k_weight, const int32_t* seqlens,
                          void* q_out, void* r_out, void* k_cache, void* v_cache, void* out, int B, int Hq, int Hkv,
@@ -1779,6 +1781,11 @@ int parallax_decode_step(const void* q_raw, const void* r_raw, const void* k_raw
     rc = parallax_decode_prepare(q_raw, r_raw, k_raw, v_raw, q_weight, r_weight, k_weight, seqlens, q_out, r_out, k_cache,
                                  v_cache, B, Hq, Hkv, D, T_max, eps, rope_theta, rope_on_r, stream);
     if (rc != PLX_OK) return rc;
+    // groups that parallax_decode_fwd_ex hands to the multi-token entry (more than eight heads per KV head, more than four
+    // at D = 128) take that route here too, as an ordinary launch behind the upstream kernel
+    if (Hq / Hkv > (D == 128 ? 4 : kMaxGroupOneCta))
+        return parallax_decode_fwd_ex(q_out, r_out, k_cache, v_cache, seqlens, out, B, Hq, Hkv, D, T_max, scale, out_dtype,
+                                      workspace, workspace_bytes, num_splits, stream);
     return decode_fwd_impl(q_out, r_out, k_cache, v_cache, seqlens, out, B, Hq, Hkv, D, T_max, scale, out_dtype, workspace,
                            workspace_bytes, num_splits, stream, nullptr, 0, 0, 0, false, 1.0f, 1.0f, true);
 }
@@ -1809,6 +1816,7 @@ int parallax_decode_fwd_fp8(const void* q, const void* r, const void* k_cache, c
 constexpr int kMultiTokenDecodeRows = PLX_MULTI_TOKEN_DECODE_ROWS;
 constexpr int kTwoCtaDecodeRows = 16;
 // rows per KV head above which a multi-token step goes to the keys-on-lanes tensor-core kernel
+static_assert(kMaxGroupOneCta == kMultiTokenDecodeRows, "parallax_decode_step mirrors the routing of parallax_decode_fwd_ex");
 static int rows_kernel_from(int D) { return D == 128 ? 4 : kMultiTokenDecodeRows; }
 // Does a step of this shape go to the keys-on-lanes kernel (given that it supports the shape)?  page_size 0: contiguous.
 // 33 to 64 rows per KV head run there as two parts that share their K/V through L2: at D = 128 that beats the row-major
@@ -1934,8 +1942,9 @@ int parallax_decode_fwd_ex(const void* q, const void* r, const void* k_cache, co
                            float scale, int out_dtype, void* workspace, size_t workspace_bytes, int num_splits,
                            void* stream)
 {
-    // more than eight query heads per KV head (multi-query models): the one-token step of the multi-token entry
-    if (Hq > 0 && Hkv > 0 && Hq % Hkv == 0 && Hq / Hkv > kMultiTokenDecodeRows)
+    // more than eight query heads per KV head (multi-query models; more than four at D = 128, where the keys-on-lanes
+    // kernel is ahead from five rows on): the one-token step of the multi-token entry
+    if (Hq > 0 && Hkv > 0 && Hq % Hkv == 0 && Hq / Hkv > rows_kernel_from(D))
         return parallax_decode_fwd_multi(q, r, k_cache, v_cache, seqlens, out, B, Hq, Hkv, D, 1, T_max, scale, out_dtype,
                                          workspace, workspace_bytes, num_splits, stream);
     return decode_fwd_impl(q, r, k_cache, v_cache, seqlens, out, B, Hq, Hkv, D, T_max, scale, out_dtype, workspace,
@@ -1948,7 +1957,7 @@ int parallax_decode_fwd_paged(const void* q, const void* r, const void* k_pages,
                               void* workspace, size_t workspace_bytes, int num_splits, void* stream)
 {
     if (!block_table) return PLX_ERR_NULL_POINTER;
-    if (Hq > 0 && Hkv > 0 && Hq % Hkv == 0 && Hq / Hkv > kMultiTokenDecodeRows)  // as in parallax_decode_fwd_ex
+    if (Hq > 0 && Hkv > 0 && Hq % Hkv == 0 && Hq / Hkv > (page_size >= 64 ? rows_kernel_from(D) : kMultiTokenDecodeRows))  // as in parallax_decode_fwd_ex
         return parallax_decode_fwd_multi_paged(q, r, k_pages, v_pages, block_table, seqlens, out, B, Hq, Hkv, D, 1,
                                                num_pages, page_size, max_pages_per_seq, scale, out_dtype, workspace,
                                                workspace_bytes, num_splits, stream);
