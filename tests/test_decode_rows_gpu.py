@@ -317,6 +317,11 @@ def test_rows_more_items_than_sms_drawn_from_the_ticket(plx, oracle, D, Lq, T, n
         assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])
         assert int(ws[:256].view(torch.int32).abs().sum().item()) == 0      # status and ticket are zero again
         assert_parity(outs[0].cpu().numpy(), want, torch.float32, f"ticket D={D} Lq={Lq} ns={ns} ragged={seqlens is not None}")
+        if ns == 1:     # without a workspace: one CTA per item, the same items, the same bits
+            out = torch.full((B, cfg.Hq, Lq, D), float("nan"), dtype=torch.float32, device="cuda")
+            plx.parallax_decode_fwd_multi(x["q"], x["r"], x["k"], x["v"], x["seqlens"], out, cfg.scale, None, 1)
+            torch.cuda.synchronize()
+            assert torch.equal(out, outs[0])
 
 
 def test_rows_ticket_walk_over_a_paged_cache_and_from_a_cuda_graph(plx, oracle):
