@@ -380,8 +380,9 @@ int parallax_decode_fwd_multi(const void* q, const void* r, const void* k_cache,
  * through L2), D = 64 or 128, bf16 caches, contiguous layout; q, r, k_cache,
  * v_cache, out 16-byte aligned.  Split-KV like parallax_prefill_fwd_ex: `workspace` holds split records only
  * (parallax_prefill_workspace_bytes(B, Hq, D, Lq, max_splits) bytes, 16-byte aligned; NULL = one split),
- * num_splits 0 = planned (about one CTA per SM, at least four 128-key tiles per split), records merged by the
- * decode path's combine kernel on the same stream.  `status` (device int32, may be NULL) receives
+ * num_splits 0 = planned (fewer items than SMs: about one CTA per SM, at least four 128-key tiles per split; more:
+ * the count a model of the step's time prefers, often 1), records merged by the decode path's merge kernels on
+ * the same stream.  `status` (device int32, may be NULL) receives
  * PLX_ERR_DEVICE_TIMEOUT if a bounded device-side wait runs out.  PLX_ERR_UNSUPPORTED for other shapes.
  * parallax_decode_fwd_multi chooses this kernel by itself (parallax_decode_fwd_multi_paged too, over paged
  * caches); this entry forces it.  Arguments, token order and causal rule as parallax_decode_fwd_multi.  One or
