@@ -187,3 +187,45 @@ def test_the_plan_query_names_the_kernel_that_runs(plx):
     assert plan(Lq=8, B=256, T=2048) == (K.PLX_MULTI_KERNEL_ROWS, 1)
     with pytest.raises(plx.ParallaxError):
         plx.parallax_decode_multi_plan(4, 5, 2, 128, 1, 4096, 0)
+
+
+@pytest.mark.parametrize("name,Lq,nrows", [("C3", 4, 512), ("C3", 8, 768), ("C3", 24, 512), ("C5", 8, 768), ("C6", 16, 512),
+                                            ("C4", 16, 256), ("C2", 8, 512)])
+def test_multi_token_full_size_in_the_bench_configuration(plx, oracle, name, Lq, nrows):
+    """The decode configurations at full size with several new tokens per sequence, in the launch configuration the
+    bench times (routed entry, planned splits, bf16 output): sampled (sequence, head, token) rows against the fp64
+    oracle of the ONE-token path on the context that token sees (token i sees the first L - (Lq - 1 - i) keys), which is
+    what the multi-token causal rule says.  Covers the item walk (C3, C5, C6), two parts of the rows (C3 with 24
+    tokens), few long streams (C4) and a grid smaller than the device (C2)."""
+    cfg = wl.CONFIGS[name]
+    x = wl.make_prefill_inputs(cfg, Lq, "cuda", poison_padding=(name == "C5"))
+    out = torch.full((cfg.B, cfg.Hq, Lq, cfg.D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    ws = plx.alloc_workspace(cfg.B, cfg.Hq * Lq, cfg.D, plx.PLX_MAX_SPLITS, "cuda")
+    plx.parallax_decode_fwd_multi(x["q"], x["r"], x["k"], x["v"], x["seqlens"], out, cfg.scale, ws, 0)
+    torch.cuda.synchronize()
+    assert plx.parallax_workspace_status(ws) == 0
+    assert torch.isfinite(out.float()).all()
+    rng = np.random.default_rng(11)
+    picks = {(0, 0, 0), (cfg.B - 1, cfg.Hq - 1, Lq - 1), (0, cfg.Hq - 1, 0)}
+    while len(picks) < nrows:
+        picks.add((int(rng.integers(cfg.B)), int(rng.integers(cfg.Hq)), int(rng.integers(Lq))))
+    picks = sorted(picks)
+    sl = x["seqlens_host"]
+    G = cfg.Hq // cfg.Hkv
+    got, want = [], []
+    for (b, h, i) in picks:
+        L = cfg.T_max if sl is None else int(sl[b])
+        Li = max(L - (Lq - 1 - i), 0)
+        got.append(out[b, h, i].float().cpu().numpy())
+        if Li == 0:
+            want.append(np.zeros(cfg.D))
+            continue
+        hkv = h // G
+        q = wl.bf16_bits(x["q"][b:b + 1, h:h + 1, i])
+        r = wl.bf16_bits(x["r"][b:b + 1, h:h + 1, i])
+        k = wl.bf16_bits(x["k"][b:b + 1, hkv:hkv + 1, :Li])
+        v = wl.bf16_bits(x["v"][b:b + 1, hkv:hkv + 1, :Li])
+        o, _ = oracle.decode_bf16(q, r, k, v, np.array([Li], dtype=np.int32), cfg.scale)
+        want.append(o[0, 0])
+    e = assert_parity(np.stack(got), np.stack(want), torch.bfloat16, f"{name} Lq={Lq}")
+    print(name, Lq, e)
