@@ -323,7 +323,7 @@ def parallax_decode_multi_plan(B, Hq, Hkv, D, Lq, T_max, page_size=0):
 
 def parallax_decode_fwd_rows(q, r, k_cache, v_cache, seqlens, out, scale, workspace=None, num_splits=0, status=None,
                              stream=None):
-    """The keys-on-lanes tensor-core kernel for a step of up to 32 rows per KV head ((Hq / Hkv) * Lq <= 32, D = 64 or 128);
+    """The keys-on-lanes tensor-core kernel for a step of up to 64 rows per KV head ((Hq / Hkv) * Lq <= 64, D = 64 or 128);
     q, r, out [B, Hq, Lq, D]; workspace: uint8 CUDA tensor of parallax_prefill_workspace_bytes(...) bytes for split
     records, or None for one split.  parallax_decode_fwd_multi picks this kernel by itself."""
     _require(q, r, k_cache, v_cache, seqlens, out, workspace, status)

@@ -1801,8 +1801,8 @@ int parallax_decode_fwd_fp8(const void* q, const void* r, const void* k_cache, c
 }
 
 // Which kernel takes a step of `rows` = (query heads per KV head) x (new tokens) rows per KV head.  Up to eight
-// rows one CTA of the decode kernel serves a KV head and is the faster route at every batch size.  Nine to 32 rows
-// go to the keys-on-lanes tensor-core kernel (parallax_decode_fwd_multi decides that before it asks here).
+// rows one CTA of the decode kernel can serve a KV head.  Five (at D = 64 nine) to 64 rows go to the keys-on-lanes
+// tensor-core kernel (rows_kernel_takes below; parallax_decode_fwd_multi decides that before it asks here).
 // For what that kernel does not serve (other page sizes, unaligned rows): nine to sixteen rows that split into two CTAs of at
 // most eight (10 = 2 x 5, 12, 14, 16) stay on the decode kernel, the rest goes to the row-major tensor-core kernel: measured
 // at 10 / 12 / 16 rows, 8 KV heads, decode kernel against the split-KV tensor-core kernel: 64 x 8192 keys 505 / 525 /
@@ -1870,7 +1870,7 @@ int parallax_decode_fwd_multi(const void* q, const void* r, const void* k_cache,
 {
     if (Lq <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || B <= 0) return PLX_ERR_BAD_SHAPE;
     if (workspace && !aligned(workspace, 16)) return PLX_ERR_ALIGNMENT;
-    // Nine to 32 rows per KV head: the tensor-core kernel with the keys on the accumulator lanes, whose work
+    // Up to 64 rows per KV head: the tensor-core kernel with the keys on the accumulator lanes, whose work
     // follows the rows present.  Measured against the routes below (D = 128, 8 KV heads, 10 / 16 / 24 / 32 rows, us per step):
     // 64 x 8192 keys 342 / 350 / 375 / 388 against 474 / 506 / 722 / 766; 16 x 8192 90 / 87 / 91 / 91 against 146 / 154 /
     // 182 / 182; 8 x 8192 53 / 53 / 57 / 58 against 80 / 87 / 116 / 107; 2 x 131072 167 / 169 / 172 / 172 against 323 / 334 /

@@ -1,4 +1,4 @@
-// Multi-token decode step with up to 32 rows per KV head (a handful to a few dozen new tokens per sequence
+// Multi-token decode step with up to 64 rows per KV head, 32 per CTA (a handful to a few dozen new tokens per sequence
 // times the query heads of a GQA group) on the tcgen05 tensor cores, with the KEYS on the TMEM lanes.
 //
 // The row-major multi-token kernel computes a 128-row tile whatever the number of rows, and the mma.sync decode
