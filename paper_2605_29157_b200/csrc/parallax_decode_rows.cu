@@ -110,7 +110,8 @@ struct RowsCfg {
     static constexpr int kOffAlpha = kOffRef + NR * 4;    // float [NR]: rescale factors of a tile that moves references
     static constexpr int kOffWmax = kOffAlpha + NR * 4;   // float [element-wise warps][RPT]: per-warp tile maxima
     static constexpr int kOffItems = kOffWmax + kEwWarps * RPT * 4;  // int [2]: the items handed from the producer to the other roles
-    static constexpr int kSmemBytes = kOffItems + 16;
+    static constexpr int kOffDsum = kOffItems + 16;  // float [element-wise warps][RPT][2] per-warp row sums, then [NR][2] totals
+    static constexpr int kSmemBytes = kOffDsum + (kEwWarps * RPT * 2 + NR * 2) * 4;
     static_assert(kSmemBytes <= 232448, "shared-memory budget of one CTA");
     static_assert(kOffK % 1024 == 0 && kOffBar % 8 == 0 && kOffRef % 16 == 0, "alignment of the tiles, barriers and references");
     static constexpr uint32_t kColS = 0;                  // two score buffers of 2 NR fp32 columns: S1^T | S2^T
@@ -536,7 +537,7 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 }
                 continue;
             }
-            // the previous item's epilogue has read the references and its scratch in the weight tile
+            // the previous item's epilogue has read the references and the row-sum scratch
             ew_barrier<kEwThreads>();
             if (threadIdx.x < NR) ref[threadIdx.x] = -INFINITY;
             ew_barrier<kEwThreads>();
@@ -739,12 +740,10 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 ROWS_T(5);
             }
 
-            // ---- row sums over the keys, then the epilogue: this thread's TMEM lane is head dimension kr ----
+            // ---- row sums over the keys (while the last value product runs), then the epilogue: this thread's TMEM lane is
+            // head dimension kr ----
             ROWS_STAMP(4);  // last weights handed over
-            wait_or_flag(bar(kBarFinal), n & 1, p.status);
-            ROWS_STAMP(5);  // last value product done
-            tc_fence_after();
-            float* const dsum = reinterpret_cast<float*>(smem + C::kOffP);  // the weight tile is idle now: [warps][RPT][2], then [NR][2]
+            float* const dsum = reinterpret_cast<float*>(smem + C::kOffDsum);
             {
                 const float t1 = warp_transpose_reduce<RPT, false>(d1, lane);
                 const float t2 = warp_transpose_reduce<RPT, false>(d2, lane);
@@ -767,6 +766,9 @@ plx_decode_rows_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 dtot[2 * row + 1] = t2;
             }
             ew_barrier<kEwThreads>();
+            wait_or_flag(bar(kBarFinal), n & 1, p.status);
+            ROWS_STAMP(5);  // last value product done
+            tc_fence_after();
             {
                 uint32_t u0[RPT], u1[RPT], w0[RPT], w1[RPT];
                 ld_cols(lane_base + C::kColO + 0 * NR + c0, u0);
